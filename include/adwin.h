@@ -1,0 +1,164 @@
+/*
+ * adwin.h -- C ABI of the B200 (sm_100a) windowed on-policy-distillation divergence library.
+ *
+ * The library evaluates, for every response position that lies inside its sequence's prefix
+ * window, the teacher-student divergence over the full vocabulary, its gradient with respect to
+ * the student logits, and the per-sequence / per-batch reductions that the prefix-versus-full
+ * alignment audit consumes (ADWIN: Adaptive Windows for Horizon-Aware On-Policy Distillation).
+ *
+ * Notation: row r = (b,t); z = student_logits[b,t,:], u = teacher_logits[b,t,:], y = tokens[b,t];
+ * p = softmax(z), q = softmax(u); W_b = window[b] (the training window L_t of Section 4.1, given
+ * per sequence), R_b = rollout_len[b]; E_b = min(W_b, R_b, T) is the effective window.  Positions
+ * are 0-based response positions; logits[b,t,:] is the distribution y[b,t] was drawn from (the
+ * library never shifts).
+ *
+ * Pointer convention: every pointer is a DEVICE pointer owned by the caller unless its comment
+ * says "host".  The library allocates nothing, frees nothing and never synchronises the stream:
+ * all work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *
+ * Errors: the int return value is an adwin_status_t detected on the host before anything is
+ * launched (nothing is enqueued on error).  Conditions that only the device can see (array
+ * contents) OR bits of adwin_dev_status_t into *dev_status; the kernels finish without faulting.
+ */
+#ifndef ADWIN_H_
+#define ADWIN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ADWIN_OK = 0,
+  ADWIN_ERR_NULL = 1,        /* a required pointer is NULL */
+  ADWIN_ERR_SHAPE = 2,       /* B, T, V, ld, K out of range */
+  ADWIN_ERR_ALIGN = 3,       /* a pointer is not aligned to its element type */
+  ADWIN_ERR_DTYPE = 4,       /* unknown dtype / grad mode / flag */
+  ADWIN_ERR_WINDOW = 5,      /* reserved for host-visible window errors */
+  ADWIN_ERR_WORKSPACE = 6,   /* workspace NULL, misaligned or smaller than adwin_workspace_bytes */
+  ADWIN_ERR_CUDA = 7,        /* a CUDA runtime call failed (launch, attribute, copy) */
+  ADWIN_ERR_UNSUPPORTED = 8  /* the requested combination is not implemented */
+} adwin_status_t;
+
+/* Bits OR-ed into *dev_status by the kernels. */
+typedef enum {
+  ADWIN_DEV_TOKEN_RANGE = 1, /* some processed tokens[b,t] outside [0,V): that row's logratio is NaN */
+  ADWIN_DEV_NONFINITE = 2,   /* a processed row produced a non-finite log-sum-exp */
+  ADWIN_DEV_TIMEOUT = 4,     /* a bounded on-chip wait ran out; outputs of this call are invalid */
+  ADWIN_DEV_BOUNDS = 8,      /* an internal index check failed; outputs of this call are invalid */
+  ADWIN_DEV_WINDOW = 16      /* some W_b < 0, R_b < 0 or R_b > T; the value was clamped to [0,T] */
+} adwin_dev_status_t;
+
+typedef enum { ADWIN_F32 = 0, ADWIN_BF16 = 1 } adwin_dtype_t;
+
+/* Which gradient estimator the call evaluates (also decides what gsq is the squared norm of). */
+typedef enum {
+  ADWIN_GRAD_FULL_KL = 0, /* g_k = alpha p_k (log p_k - log q_k - KL): d/dz of the per-token reverse
+                             KL(p||q), the full-vocabulary form of the OPD objective (Eq. 2) */
+  ADWIN_GRAD_SAMPLED = 1  /* g_k = alpha c (1[k=y] - p_k): the gamma=0 token-local estimator
+                             c_t * d log pi_theta(y_t) / dz (Eq. 4), c held constant */
+} adwin_grad_mode_t;
+
+enum {
+  ADWIN_ZERO_TAIL = 1,     /* zero-fill gradient rows t >= E_b instead of leaving them untouched */
+  ADWIN_RANGE_FULL = 2,    /* per-token scalars for every t < R_b (delayed full-rollout probe,
+                              Section 4.2); the gradient is still written only for t < E_b */
+  ADWIN_FORCE_GENERIC = 4  /* use the shape-agnostic kernel even when the staged kernel applies */
+};
+
+/* Flags returned by adwin_probe_align in *flags_out. */
+enum {
+  ADWIN_ALIGN_DEGENERATE = 1,      /* some full-rollout squared norm was 0: that rho was set to 1 */
+  ADWIN_ALIGN_NONE_ADMISSIBLE = 2  /* no candidate reached rho_star: L_next = largest candidate */
+};
+
+/* Library ABI version (bumped when a signature changes). */
+int adwin_version(void);
+
+/* Human-readable name of an adwin_status_t.  Host pointer to a static string. */
+const char* adwin_status_string(int status);
+
+/*
+ * Bytes of device scratch that adwin_opd_kl_fwd_bwd needs for these shapes (the in-window row map:
+ * effective ranges and their prefix sums).  Always > 0; the buffer must be 256-byte aligned.
+ */
+size_t adwin_workspace_bytes(int64_t B, int64_t T, int64_t V, int dtype, int flags);
+
+/*
+ * Windowed per-token OPD divergence, forward and backward, one pass over the logits.
+ *
+ * For every processed row (t < E_b; with ADWIN_RANGE_FULL: t < R_b) it computes, with fp32
+ * accumulation,
+ *   lse_s = log sum_k exp z_k, lse_t = log sum_k exp u_k        (log-softmax normalisers)
+ *   kl[b,t]       = sum_k p_k (log p_k - log q_k)               reverse KL(p||q), per-token form of
+ *                                                               the OPD objective (Eq. 2)
+ *   logratio[b,t] = log p_y - log q_y                           step-wise cost c_t (Section 2.3);
+ *                                                               the token reward is -c_t (App. A.1)
+ *   gsq[b,t]      = sum_k g_k^2                                 squared norm of the row's gradient
+ * and, when grad_student != NULL and t < E_b, writes g (see adwin_grad_mode_t, alpha = grad_scale)
+ * to grad_student[b,t,:].  Rows past the window are skipped entirely: their logits are never read
+ * and their gradient rows are left untouched (or zero-filled with ADWIN_ZERO_TAIL).  Per-token
+ * outputs of rows that are not processed are written as 0.
+ *
+ * student_logits, teacher_logits : [B,T,V], element type `dtype`, row stride `ld` elements
+ *                                  (row r = b*T+t starts at element r*ld; ld >= V)
+ * tokens       : [B,T] int32            window : [B] int32
+ * rollout_len  : [B] int32 or NULL (= T for every sequence)
+ * grad_student : [B,T,V] of `grad_dtype`, row stride ld_grad, or NULL (no gradient is written;
+ *                gsq is then accumulated in the same single sweep)
+ * kl, logratio : [B,T] fp32, required.   gsq, lse_student, lse_teacher : [B,T] fp32 or NULL
+ * workspace    : >= adwin_workspace_bytes(...) bytes, 256-byte aligned; contents undefined after
+ * dev_status   : one int32 the caller zeroed; bits are OR-ed in
+ *
+ * The staged (fast) kernel needs 16-byte aligned logits / gradient base pointers, row strides
+ * that are multiples of 16 bytes and V*sizeof(element) a multiple of 16; any other layout runs
+ * through the shape-agnostic kernel with identical results up to rounding order.
+ */
+int adwin_opd_kl_fwd_bwd(const void* student_logits, const void* teacher_logits, int dtype,
+                         int64_t B, int64_t T, int64_t V, int64_t ld, const int32_t* tokens,
+                         const int32_t* window, const int32_t* rollout_len, float grad_scale,
+                         int grad_mode, int flags, void* grad_student, int grad_dtype,
+                         int64_t ld_grad, float* kl, float* logratio, float* gsq,
+                         float* lse_student, float* lse_teacher, void* workspace,
+                         size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
+
+/*
+ * Windowed sums: the loss "on this prefix" that the synchronous update uses (Section 4.1).
+ * seq_out[b] = { sum_{t<E_b} kl, sum_{t<E_b} logratio, sum_{t<E_b} gsq, E_b } and batch_out =
+ * the same four summed over b, all in float64 with a fixed summation order (bitwise
+ * reproducible).  gsq may be NULL (its sums are 0).  seq_out [B,4], batch_out [4]: device.
+ */
+int adwin_window_reduce(const float* kl, const float* logratio, const float* gsq,
+                        const int32_t* window, const int32_t* rollout_len, int64_t B, int64_t T,
+                        double* seq_out, double* batch_out, void* cuda_stream);
+
+/*
+ * Prefix-versus-full alignment audit on a returned probe batch (Section 4.2), in logit space.
+ * Input: per-token scalars valid on t < R_b (a call with ADWIN_RANGE_FULL).  In logit space the
+ * prefix gradient is the full-rollout gradient with rows t >= L zeroed, hence
+ *   rho(L) = cos(u_probe, u^(L)) = sqrt(Q(L)/Q_full),   Q(L) = sum_{t < min(L,R_b)} gsq[b,t].
+ * Slots j = 0..K-1 are the candidate lengths, slot K is each sequence's own W_b.
+ *   seq_stats   [B,K+1,4] = { Q_b(L_j), sum kl, sum logratio over the same prefix, rho_b(L_j) }
+ *   seq_full    [B,3]     = { Q_b_full, sum kl, sum logratio over t < R_b }
+ *   batch_stats [K+1,5]   = { rho_micro, rho_macro, snr_micro, admissible (0/1), n_tokens }
+ * rho_macro = mean over the B sequences of rho_b; rho_micro = the cosine after batch aggregation
+ * (Figure 5); SNR = rho^2/(1-rho^2); admissible <=> rho_micro >= rho_star (Eq. 5, inclusive).
+ * *L_next = the smallest admissible candidate (the scheduler rule of Section 4.2), or the largest
+ * candidate with ADWIN_ALIGN_NONE_ADMISSIBLE.  A zero full norm gives rho = 1 and
+ * ADWIN_ALIGN_DEGENERATE.
+ * candidates : [K] int32 DEVICE pointer, or NULL for the paper's list {64,...,2048} (then K must
+ *              be 0 or 6).  1 <= K <= 64.     rho_star <= 0 selects sqrt(2)/2.
+ * All outputs are device pointers (float64 / int32), summed in a fixed order.
+ */
+int adwin_probe_align(const float* kl, const float* logratio, const float* gsq,
+                      const int32_t* window, const int32_t* rollout_len, int64_t B, int64_t T,
+                      const int32_t* candidates, int32_t K, double rho_star, double* seq_stats,
+                      double* seq_full, double* batch_stats, int32_t* L_next, int32_t* flags_out,
+                      void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADWIN_H_ */
