@@ -1,0 +1,183 @@
+"""ctypes binding of the C ABI declared in ``include/adwin.h``: argument marshalling only.
+
+Every step of the path runs in the CUDA library.  torch supplies device memory and the stream.
+There is no CPU fallback: if the shared library is missing the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+from pathlib import Path
+from types import SimpleNamespace
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libadwin_b200.so"
+
+OK = 0
+F32, BF16 = 0, 1
+GRAD_FULL_KL, GRAD_SAMPLED = 0, 1
+ZERO_TAIL, RANGE_FULL, FORCE_GENERIC = 1, 2, 4
+DEV_TOKEN_RANGE, DEV_NONFINITE, DEV_TIMEOUT, DEV_BOUNDS, DEV_WINDOW = 1, 2, 4, 8, 16
+ALIGN_DEGENERATE, ALIGN_NONE_ADMISSIBLE = 1, 2
+DEFAULT_CANDIDATES = (64, 128, 256, 512, 1024, 2048)   # Section 5.1, Training Details
+RHO_STAR = math.sqrt(2.0) / 2.0                          # Eq. 5
+
+EXPORTS = ("adwin_version", "adwin_status_string", "adwin_workspace_bytes",
+           "adwin_opd_kl_fwd_bwd", "adwin_window_reduce", "adwin_probe_align")
+
+_lib = None
+
+
+class AdwinError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__(lib().adwin_status_string(code).decode())
+
+
+def lib():
+    """Load libadwin_b200.so (built by ``build.py``); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2605_28396_b200.build`; "
+                "there is no fallback path")
+        L = ctypes.CDLL(str(LIB_PATH))
+        vp, i64, i32, f32, f64, sz = (ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32,
+                                      ctypes.c_float, ctypes.c_double, ctypes.c_size_t)
+        L.adwin_version.restype = ctypes.c_int
+        L.adwin_status_string.restype = ctypes.c_char_p
+        L.adwin_status_string.argtypes = [ctypes.c_int]
+        L.adwin_workspace_bytes.restype = sz
+        L.adwin_workspace_bytes.argtypes = [i64, i64, i64, ctypes.c_int, ctypes.c_int]
+        L.adwin_opd_kl_fwd_bwd.restype = ctypes.c_int
+        L.adwin_opd_kl_fwd_bwd.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, i64, vp, vp, vp,
+                                           f32, ctypes.c_int, ctypes.c_int, vp, ctypes.c_int, i64,
+                                           vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.adwin_window_reduce.restype = ctypes.c_int
+        L.adwin_window_reduce.argtypes = [vp, vp, vp, vp, vp, i64, i64, vp, vp, vp]
+        L.adwin_probe_align.restype = ctypes.c_int
+        L.adwin_probe_align.argtypes = [vp, vp, vp, vp, vp, i64, i64, vp, i32, f64, vp, vp, vp,
+                                        vp, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(device):
+    return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+def _dtype_code(dt):
+    if dt == torch.float32:
+        return F32
+    if dt == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {dt}")
+
+
+def _check(rc):
+    if rc != OK:
+        raise AdwinError(rc)
+
+
+def adwin_workspace_bytes(B, T, V, dtype=BF16, flags=0) -> int:
+    return int(lib().adwin_workspace_bytes(B, T, V, dtype, flags))
+
+
+def adwin_opd_kl_fwd_bwd(student, teacher, tokens, window, rollout_len=None, *, grad_scale=1.0,
+                         grad_mode=GRAD_FULL_KL, flags=0, grad=None, grad_dtype=None,
+                         want_gsq=True, want_lse=False, out=None, workspace=None, dev_status=None):
+    """Windowed per-token OPD divergence, forward + backward (see include/adwin.h).
+
+    student, teacher: [B,T,V] CUDA tensors (fp32 or bf16), last dim contiguous, rows at a uniform
+    stride.  ``grad``: a [B,T,V] tensor to write into, or None with ``grad_dtype`` set to have one
+    allocated (uninitialised outside the window unless ZERO_TAIL), or both None for no gradient.
+    Returns a namespace with kl, logratio, gsq, lse_s, lse_t, grad, dev_status (device tensors).
+    Nothing is synchronised; read ``dev_status`` (or call ``raise_on_dev_status``) after a sync.
+    """
+    assert student.is_cuda and teacher.is_cuda and student.shape == teacher.shape
+    assert student.dim() == 3 and student.dtype == teacher.dtype
+    B, T, V = student.shape
+    dev = student.device
+
+    def row_stride(x):
+        assert x.stride(2) == 1 or V == 1, "last dim must be contiguous"
+        ld = x.stride(1) if T > 1 else (x.stride(0) if B > 1 else V)
+        assert B <= 1 or T <= 1 or x.stride(0) == T * ld, "rows must sit at one uniform stride"
+        return ld
+
+    ld = row_stride(student)
+    assert row_stride(teacher) == ld, "student and teacher must share the row stride"
+    if grad is None and grad_dtype is not None:
+        grad = torch.empty((B, T, V), dtype=grad_dtype, device=dev)
+    ld_grad = row_stride(grad) if grad is not None else 0
+    o = out if out is not None else SimpleNamespace()
+    f32 = dict(dtype=torch.float32, device=dev)
+    if getattr(o, "kl", None) is None:
+        o.kl = torch.empty((B, T), **f32)
+        o.logratio = torch.empty((B, T), **f32)
+        o.gsq = torch.empty((B, T), **f32) if want_gsq else None
+        o.lse_s = torch.empty((B, T), **f32) if want_lse else None
+        o.lse_t = torch.empty((B, T), **f32) if want_lse else None
+    o.grad = grad
+    wsb = adwin_workspace_bytes(B, T, V, _dtype_code(student.dtype), flags)
+    if workspace is None:
+        workspace = torch.empty(wsb, dtype=torch.uint8, device=dev)
+    if dev_status is None:
+        dev_status = torch.zeros(1, dtype=torch.int32, device=dev)
+    o.dev_status = dev_status
+    o.workspace = workspace
+    rc = lib().adwin_opd_kl_fwd_bwd(
+        _ptr(student), _ptr(teacher), _dtype_code(student.dtype), B, T, V, ld, _ptr(tokens),
+        _ptr(window), _ptr(rollout_len), float(grad_scale), int(grad_mode), int(flags), _ptr(grad),
+        _dtype_code(grad.dtype) if grad is not None else 0, ld_grad, _ptr(o.kl), _ptr(o.logratio),
+        _ptr(o.gsq), _ptr(o.lse_s), _ptr(o.lse_t), _ptr(workspace), workspace.numel(),
+        _ptr(dev_status), _stream(dev))
+    _check(rc)
+    return o
+
+
+def raise_on_dev_status(dev_status, allow=0):
+    """Synchronising read of the device status word; raises on bits outside ``allow``."""
+    bits = int(dev_status.item())
+    if bits & ~allow:
+        names = {1: "TOKEN_RANGE", 2: "NONFINITE", 4: "TIMEOUT", 8: "BOUNDS", 16: "WINDOW"}
+        raise RuntimeError("adwin device status: " +
+                           "|".join(n for b, n in names.items() if bits & b))
+    return bits
+
+
+def adwin_window_reduce(kl, logratio, gsq, window, rollout_len=None):
+    """Per-sequence and per-batch windowed sums: returns (seq_out [B,4], batch_out [4]) float64."""
+    B, T = kl.shape
+    dev = kl.device
+    seq = torch.empty((B, 4), dtype=torch.float64, device=dev)
+    batch = torch.empty(4, dtype=torch.float64, device=dev)
+    _check(lib().adwin_window_reduce(_ptr(kl), _ptr(logratio), _ptr(gsq), _ptr(window),
+                                     _ptr(rollout_len), B, T, _ptr(seq), _ptr(batch),
+                                     _stream(dev)))
+    return seq, batch
+
+
+def adwin_probe_align(kl, logratio, gsq, window, rollout_len=None, candidates=None, rho_star=0.0):
+    """Prefix-versus-full alignment audit.  ``candidates``: int32 CUDA tensor or None (paper list)."""
+    B, T = kl.shape
+    dev = kl.device
+    K = 6 if candidates is None else int(candidates.numel())
+    f64 = dict(dtype=torch.float64, device=dev)
+    o = SimpleNamespace(
+        seq_stats=torch.empty((B, K + 1, 4), **f64), seq_full=torch.empty((B, 3), **f64),
+        batch_stats=torch.empty((K + 1, 5), **f64),
+        L_next=torch.zeros(1, dtype=torch.int32, device=dev),
+        flags=torch.zeros(1, dtype=torch.int32, device=dev))
+    _check(lib().adwin_probe_align(_ptr(kl), _ptr(logratio), _ptr(gsq), _ptr(window),
+                                   _ptr(rollout_len), B, T, _ptr(candidates), K, float(rho_star),
+                                   _ptr(o.seq_stats), _ptr(o.seq_full), _ptr(o.batch_stats),
+                                   _ptr(o.L_next), _ptr(o.flags), _stream(dev)))
+    return o

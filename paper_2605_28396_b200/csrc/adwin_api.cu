@@ -1,0 +1,181 @@
+// extern "C" entry points: argument validation and kernel dispatch.  No allocation, no
+// synchronisation; everything is enqueued on the caller's stream.
+#include <mutex>
+
+#include "adwin_common.cuh"
+#include "adwin_internal.h"
+
+namespace adwin {
+namespace {
+
+constexpr int kKnownFlags = ADWIN_ZERO_TAIL | ADWIN_RANGE_FULL | ADWIN_FORCE_GENERIC;
+constexpr int64_t kMaxB = int64_t(1) << 24;
+constexpr int64_t kMaxT = int64_t(1) << 24;
+constexpr int64_t kMaxV = int64_t(1) << 28;
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline size_t elem_size(int dtype) { return dtype == ADWIN_F32 ? 4 : 2; }
+
+int sm_count_of_current_device() {
+  static std::mutex mu;
+  static int cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+  std::lock_guard<std::mutex> lock(mu);
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      return -1;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+}  // namespace
+}  // namespace adwin
+
+using namespace adwin;
+
+extern "C" {
+
+int adwin_version(void) { return 1; }
+
+const char* adwin_status_string(int status) {
+  switch (status) {
+    case ADWIN_OK: return "ADWIN_OK";
+    case ADWIN_ERR_NULL: return "ADWIN_ERR_NULL: a required pointer is NULL";
+    case ADWIN_ERR_SHAPE: return "ADWIN_ERR_SHAPE: a dimension or stride is out of range";
+    case ADWIN_ERR_ALIGN: return "ADWIN_ERR_ALIGN: a pointer is not aligned to its element type";
+    case ADWIN_ERR_DTYPE: return "ADWIN_ERR_DTYPE: unknown dtype, gradient mode or flag";
+    case ADWIN_ERR_WINDOW: return "ADWIN_ERR_WINDOW: invalid window or rollout length";
+    case ADWIN_ERR_WORKSPACE: return "ADWIN_ERR_WORKSPACE: workspace missing, misaligned or too small";
+    case ADWIN_ERR_CUDA: return "ADWIN_ERR_CUDA: a CUDA runtime call failed";
+    case ADWIN_ERR_UNSUPPORTED: return "ADWIN_ERR_UNSUPPORTED: combination not implemented";
+    default: return "unknown adwin status";
+  }
+}
+
+size_t adwin_workspace_bytes(int64_t B, int64_t T, int64_t V, int dtype, int flags) {
+  (void)T; (void)V; (void)dtype; (void)flags;
+  if (B < 0) B = 0;
+  return workspace_layout(B).total;
+}
+
+int adwin_opd_kl_fwd_bwd(const void* student_logits, const void* teacher_logits, int dtype,
+                         int64_t B, int64_t T, int64_t V, int64_t ld, const int32_t* tokens,
+                         const int32_t* window, const int32_t* rollout_len, float grad_scale,
+                         int grad_mode, int flags, void* grad_student, int grad_dtype,
+                         int64_t ld_grad, float* kl, float* logratio, float* gsq,
+                         float* lse_student, float* lse_teacher, void* workspace,
+                         size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+  if (dtype != ADWIN_F32 && dtype != ADWIN_BF16) return ADWIN_ERR_DTYPE;
+  if (grad_mode != ADWIN_GRAD_FULL_KL && grad_mode != ADWIN_GRAD_SAMPLED) return ADWIN_ERR_DTYPE;
+  if (flags & ~kKnownFlags) return ADWIN_ERR_DTYPE;
+  if (grad_student && grad_dtype != ADWIN_F32 && grad_dtype != ADWIN_BF16) return ADWIN_ERR_DTYPE;
+  if (B < 0 || T < 0 || B > kMaxB || T > kMaxT || V < 1 || V > kMaxV || ld < V)
+    return ADWIN_ERR_SHAPE;
+  if (grad_student && ld_grad < V) return ADWIN_ERR_SHAPE;
+  if (!dev_status) return ADWIN_ERR_NULL;
+  if (B == 0 || T == 0) return ADWIN_OK;
+  if (!student_logits || !teacher_logits || !tokens || !window || !kl || !logratio)
+    return ADWIN_ERR_NULL;
+  const size_t es = elem_size(dtype);
+  if (!aligned(student_logits, es) || !aligned(teacher_logits, es) || !aligned(tokens, 4) ||
+      !aligned(window, 4) || !aligned(rollout_len, 4) || !aligned(kl, 4) ||
+      !aligned(logratio, 4) || !aligned(gsq, 4) || !aligned(lse_student, 4) ||
+      !aligned(lse_teacher, 4) || !aligned(dev_status, 4))
+    return ADWIN_ERR_ALIGN;
+  if (grad_student && !aligned(grad_student, elem_size(grad_dtype))) return ADWIN_ERR_ALIGN;
+  if (!workspace || !aligned(workspace, 256) ||
+      workspace_bytes < adwin_workspace_bytes(B, T, V, dtype, flags))
+    return ADWIN_ERR_WORKSPACE;
+  const int sms = sm_count_of_current_device();
+  if (sms <= 0) return ADWIN_ERR_CUDA;
+
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const WorkspaceLayout wl = workspace_layout(B);
+  char* wbase = static_cast<char*>(workspace);
+
+  KlParams p;
+  p.student = student_logits;
+  p.teacher = teacher_logits;
+  p.B = B; p.T = T; p.V = V; p.ld = ld;
+  p.tokens = tokens;
+  p.alpha = grad_scale;
+  p.mode = grad_mode;
+  p.flags = flags;
+  p.grad = grad_student;
+  p.ld_grad = grad_student ? ld_grad : 0;
+  p.kl = kl; p.logratio = logratio; p.gsq = gsq; p.lse_s = lse_student; p.lse_t = lse_teacher;
+  p.status = dev_status;
+  p.offsets = reinterpret_cast<const int64_t*>(wbase + wl.off_offsets);
+  p.range = reinterpret_cast<const int32_t*>(wbase + wl.off_range);
+  p.ewin = reinterpret_cast<const int32_t*>(wbase + wl.off_ewin);
+
+  if (launch_rowmap(window, rollout_len, B, T, flags, workspace, kl, logratio, gsq, lse_student,
+                    lse_teacher, dev_status, s) != cudaSuccess)
+    return ADWIN_ERR_CUDA;
+  if ((flags & ADWIN_ZERO_TAIL) && grad_student) {
+    if (launch_zero_tail(p, grad_dtype, s) != cudaSuccess) return ADWIN_ERR_CUDA;
+  }
+
+  // 16-byte layout test shared by the vectorised generic path and the staged kernel.
+  const int gd = grad_student ? grad_dtype : dtype;
+  bool vec16 = aligned(student_logits, 16) && aligned(teacher_logits, 16) &&
+               (ld * es) % 16 == 0 && (V * es) % 16 == 0;
+  if (grad_student)
+    vec16 = vec16 && aligned(grad_student, 16) && (ld_grad * elem_size(gd)) % 16 == 0 &&
+            (V * elem_size(gd)) % 16 == 0;
+
+  if (vec16 && !(flags & ADWIN_FORCE_GENERIC)) {
+    const cudaError_t e = launch_kl_staged(p, dtype, gd, sms, s);
+    if (e == cudaSuccess) return ADWIN_OK;
+    if (e != cudaErrorNotSupported) return ADWIN_ERR_CUDA;
+  }
+  if (launch_kl_generic(p, dtype, gd, vec16, sms, s) != cudaSuccess) return ADWIN_ERR_CUDA;
+  return ADWIN_OK;
+}
+
+int adwin_window_reduce(const float* kl, const float* logratio, const float* gsq,
+                        const int32_t* window, const int32_t* rollout_len, int64_t B, int64_t T,
+                        double* seq_out, double* batch_out, void* cuda_stream) {
+  if (B < 0 || T < 0 || B > kMaxB || T > kMaxT) return ADWIN_ERR_SHAPE;
+  if (!batch_out) return ADWIN_ERR_NULL;
+  if (B > 0 && (!kl || !logratio || !window || !seq_out)) return ADWIN_ERR_NULL;
+  if (!aligned(kl, 4) || !aligned(logratio, 4) || !aligned(gsq, 4) || !aligned(window, 4) ||
+      !aligned(rollout_len, 4) || !aligned(seq_out, 8) || !aligned(batch_out, 8))
+    return ADWIN_ERR_ALIGN;
+  if (launch_window_reduce(kl, logratio, gsq, window, rollout_len, B, T, seq_out, batch_out,
+                           static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return ADWIN_ERR_CUDA;
+  return ADWIN_OK;
+}
+
+int adwin_probe_align(const float* kl, const float* logratio, const float* gsq,
+                      const int32_t* window, const int32_t* rollout_len, int64_t B, int64_t T,
+                      const int32_t* candidates, int32_t K, double rho_star, double* seq_stats,
+                      double* seq_full, double* batch_stats, int32_t* L_next, int32_t* flags_out,
+                      void* cuda_stream) {
+  if (B < 0 || T < 0 || B > kMaxB || T > kMaxT) return ADWIN_ERR_SHAPE;
+  if (!candidates) {
+    if (K != 0 && K != 6) return ADWIN_ERR_SHAPE;
+    K = 6;
+  }
+  if (K < 1 || K > 64) return ADWIN_ERR_SHAPE;
+  if (!batch_stats || !L_next || !flags_out) return ADWIN_ERR_NULL;
+  if (B > 0 && (!kl || !logratio || !gsq || !window || !seq_stats || !seq_full))
+    return ADWIN_ERR_NULL;
+  if (!aligned(kl, 4) || !aligned(logratio, 4) || !aligned(gsq, 4) || !aligned(window, 4) ||
+      !aligned(rollout_len, 4) || !aligned(candidates, 4) || !aligned(seq_stats, 8) ||
+      !aligned(seq_full, 8) || !aligned(batch_stats, 8) || !aligned(L_next, 4) ||
+      !aligned(flags_out, 4))
+    return ADWIN_ERR_ALIGN;
+  if (!(rho_star > 0.0)) rho_star = 0.70710678118654752440;  // sqrt(2)/2
+  if (launch_probe_align(kl, logratio, gsq, window, rollout_len, B, T, candidates, K, rho_star,
+                         seq_stats, seq_full, batch_stats, L_next, flags_out,
+                         static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return ADWIN_ERR_CUDA;
+  return ADWIN_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,43 @@
+// Host-side declarations shared by the translation units of the library (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/adwin.h"
+
+namespace adwin {
+
+struct KlParams;
+
+// Workspace layout: [0,256) reserved counters; offsets (B+1) int64; range B int32; ewin B int32.
+struct WorkspaceLayout {
+  size_t off_offsets, off_range, off_ewin, total;
+};
+WorkspaceLayout workspace_layout(int64_t B);
+
+cudaError_t launch_rowmap(const int32_t* window, const int32_t* rollout_len, int64_t B, int64_t T,
+                          int flags, void* workspace, float* kl, float* logratio, float* gsq,
+                          float* lse_s, float* lse_t, int32_t* status, cudaStream_t s);
+
+cudaError_t launch_zero_tail(const KlParams& p, int grad_dtype, cudaStream_t s);
+
+cudaError_t launch_kl_generic(const KlParams& p, int dtype, int grad_dtype, bool vec, int sm_count,
+                              cudaStream_t s);
+
+// Staged cluster kernel.  Returns cudaErrorNotSupported when the shape does not fit its plan
+// (the caller then falls back to the generic kernel).
+cudaError_t launch_kl_staged(const KlParams& p, int dtype, int grad_dtype, int sm_count,
+                             cudaStream_t s);
+
+cudaError_t launch_window_reduce(const float* kl, const float* logratio, const float* gsq,
+                                 const int32_t* window, const int32_t* rollout_len, int64_t B,
+                                 int64_t T, double* seq_out, double* batch_out, cudaStream_t s);
+
+cudaError_t launch_probe_align(const float* kl, const float* logratio, const float* gsq,
+                               const int32_t* window, const int32_t* rollout_len, int64_t B,
+                               int64_t T, const int32_t* candidates, int32_t K, double rho_star,
+                               double* seq_stats, double* seq_full, double* batch_stats,
+                               int32_t* L_next, int32_t* flags_out, cudaStream_t s);
+
+}  // namespace adwin
