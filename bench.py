@@ -1,0 +1,382 @@
+#!/usr/bin/env python
+"""Benchmark of the windowed OPD divergence hot path (one JSON line on stdout).
+
+A step = one pass of the whole path over one synthetic batch: row map, the staged fwd+bwd kernel
+(log-sum-exp of both rows, reverse KL, sampled-token log-ratio, gradient, window skip), the
+windowed reductions and the alignment audit.  The workload is config 3 of the paper-shaped
+recipes in ``paper_2605_28396_b200/synth.py`` (Qwen3-scale vocabulary, reasoning-length rollouts).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 is launched with torch.distributed.run; every rank processes its own batch (weak scaling,
+no data-path collective: rows are independent) and the time is the max over ranks.
+`--impl reference` times the float64 CPU oracle, as it stands, on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+METRIC = "windowed OPD KL fwd+bwd tokens/s at V=151936"
+UNIT = "tokens/s"
+WORKLOAD = ("config3: B=16 T=2048 V=151936 bf16 logits (student N(0,4)+10*Bern(0.05), teacher = "
+            "student+N(0,2)), W_b in {256,512,1024,2048} x4, tokens ~ student softmax, "
+            "FULL_KL gradient stored bf16, rows past the window skipped")
+LAUNCHES_PER_STEP = 7   # rowmap, staged kernel, 2 window-reduce kernels, 3 audit kernels
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--seqs", type=int, default=None, help="override B (debugging only)")
+    return ap.parse_args()
+
+
+def measured_peak():
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        try:
+            return float(json.loads(f.read_text())["hbm_gbs"]), "MEASURED_PEAKS.json hbm_gbs (of measured)"
+        except Exception:
+            pass
+    return 6650.0, "fallback 6.65 TB/s (of fallback)"
+
+
+def recorded_traffic():
+    """DRAM bytes per launch from the committed ncu summary, scaled by rows (traffic is linear in rows)."""
+    f = ROOT / "profiles" / "traffic.json"
+    if f.exists():
+        try:
+            return json.loads(f.read_text())
+        except Exception:
+            return None
+    return None
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        mhz, mx, reasons, power = [], None, set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                mhz.append(float(r[0]))
+                mx = float(r[1])
+                power.append(float(r[2]))
+                for n, v in zip(names, r[4:8]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                continue
+        return {"sm_mhz": statistics.median(mhz) if mhz else None, "sm_max_mhz": mx,
+                "power_w_max": max(power) if power else None, "samples": len(mhz),
+                "reasons": sorted(reasons)}
+
+
+def oracle_sample(batch_cpu_rows):
+    """Time the oracle, as it stands, on host copies of sample rows. Returns (rows, seconds)."""
+    from oracle import adwin_oracle as O
+    s, t, tok, win = batch_cpu_rows
+    t0 = time.perf_counter()
+    O.opd_kl_fwd_bwd(s, t, tok, win, None, want_grad=True)
+    return int(win.sum()), time.perf_counter() - t0, O.num_threads()
+
+
+def sample_rows_for_oracle(batch, seqs, rows):
+    """Host copies of the first `rows` window rows of the given sequences (bf16 bits)."""
+    import numpy as np
+    import torch
+    from paper_2605_28396_b200 import synth
+    s = synth.bits_for_oracle(batch.student[seqs, :rows])
+    t = synth.bits_for_oracle(batch.teacher[seqs, :rows])
+    tok = batch.tokens[seqs, :rows].cpu().numpy()
+    win = np.minimum(batch.window[seqs].cpu().numpy(), rows).astype(np.int32)
+    return s, t, tok, win
+
+
+def run_reference(args):
+    """The reference arm of this tier: the CPU oracle on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    from paper_2605_28396_b200 import synth
+    B = 2
+    rows = 96
+    batch = synth.make_batch(3, device="cpu", B=B, T=rows)     # same recipe, bounded sample
+    batch.window[:] = rows
+    sample = sample_rows_for_oracle(batch, list(range(B)), rows)
+    for _ in range(max(0, min(args.warmup, 1))):
+        oracle_sample(sample)
+    times, n, cores = [], 0, 1
+    for _ in range(args.steps):
+        n, dt, cores = oracle_sample(sample)
+        times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    val = n / (ms / 1e3)
+    desc = f"{B} sequences x {rows} in-window rows of config 3 (V=151936) per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": desc},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": desc},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def _register(rt, view):
+    rc = rt.cudaHostRegister(view.data_ptr(), view.numel() * view.element_size(), 0)
+    if int(rc) != 0:
+        raise RuntimeError(f"cudaHostRegister failed with {rc}")
+
+
+def pinned_window_rows(batch, grad_dtype):
+    """Host images of the batch in pageable memory with only the in-window row ranges pinned
+    (rows past the window are never touched, so they are never made resident)."""
+    import torch
+    B, T, V = batch.shape
+    rt = torch.cuda.cudart()
+    host = {}
+    for name, src in (("student", batch.student), ("teacher", batch.teacher)):
+        h = torch.empty((B, T, V), dtype=src.dtype)
+        for b in range(B):
+            e = int(batch.window[b])
+            if e > 0:
+                view = h[b, :e]
+                _register(rt, view)
+                view.copy_(src[b, :e])
+        host[name] = h
+    g = torch.empty((B, T, V), dtype=grad_dtype)
+    for b in range(B):
+        e = int(batch.window[b])
+        if e > 0:
+            view = g[b, :e]
+            _register(rt, view)
+    host["grad"] = g
+    host["tokens"] = batch.tokens.cpu().pin_memory()
+    host["window"] = batch.window.cpu()
+    host["rollout_len"] = batch.rollout_len.cpu()
+    return host
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2605_28396_b200 import api, build, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    build.build()
+    api.lib()
+
+    batch = synth.make_batch(3, device=dev, seed=synth.SEED_BASE + 100000 * rank, B=args.seqs)
+    B, T, V = batch.shape
+    win_h = torch.minimum(batch.window, batch.rollout_len).cpu()
+    rows = int(win_h.sum())
+    grad = torch.empty((B, T, V), dtype=torch.bfloat16, device=dev)
+    ws = torch.empty(api.adwin_workspace_bytes(B, T, V), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    out = None
+    kl_events = []
+
+    def step(record=False):
+        nonlocal out
+        if record:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        out = api.adwin_opd_kl_fwd_bwd(batch.student, batch.teacher, batch.tokens, batch.window,
+                                       batch.rollout_len, grad=grad, out=out, workspace=ws,
+                                       dev_status=status)
+        if record:
+            e1.record()
+            kl_events.append((e0, e1))
+        seq, tot = api.adwin_window_reduce(out.kl, out.logratio, out.gsq, batch.window,
+                                           batch.rollout_len)
+        # the audit on what this pass produced: candidate prefixes against the window itself
+        al = api.adwin_probe_align(out.kl, out.logratio, out.gsq, batch.window, batch.window)
+        return tot, al
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        tot, al = step(record=True)
+    t1.record()
+    barrier()
+    ms_total = t0.elapsed_time(t1)
+    kernel_ms = statistics.mean(a.elapsed_time(b) for a, b in kl_events)
+    clocks = sampler.stop() if rank == 0 else None
+    bits = int(status.item())
+    if bits:
+        raise SystemExit(f"device status {bits}: the timed run is invalid")
+    loss = float(tot[0].item())
+
+    t = torch.tensor([ms_total, kernel_ms], dtype=torch.float64, device=dev)
+    r = torch.tensor([float(rows)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(r, op=dist.ReduceOp.SUM)
+    ms_total, kernel_ms = float(t[0]), float(t[1])
+    rows_all = float(r[0])
+    ms_step = ms_total / args.steps
+    value = rows_all / (ms_step / 1e3)
+
+    # ---- end to end through the host-buffer entry point (copies inside the timed region)
+    e2e = None
+    if not args.no_e2e:
+        host = pinned_window_rows(batch, torch.bfloat16)
+        rps = 256
+        staging = torch.empty(api.adwin_host_staging_bytes(rps, V, api.BF16, api.BF16, True),
+                              dtype=torch.uint8, device=dev)
+        hout = None
+
+        def host_step():
+            nonlocal hout
+            hout = api.adwin_opd_kl_fwd_bwd_host(host["student"], host["teacher"], host["tokens"],
+                                                 host["window"], host["rollout_len"], device=dev,
+                                                 grad=host["grad"], rows_per_stage=rps,
+                                                 staging=staging, dev_status=status, out=hout)
+        host_step()
+        barrier()
+        h0 = time.perf_counter()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.e2e_steps):
+            host_step()
+        e1.record()
+        barrier()
+        wall = (time.perf_counter() - h0) * 1e3
+        ems = max(e0.elapsed_time(e1), wall) / args.e2e_steps
+        et = torch.tensor([ems], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(et, op=dist.ReduceOp.MAX)
+        ems = float(et[0])
+        h2d = rows * V * 2 * 2 + rows * 4
+        d2h = rows * V * 2 + 3 * rows * 4
+        same = bool(torch.allclose(hout.kl, out.kl.cpu(), rtol=1e-5, atol=1e-6))
+        e2e = {"value": rows_all / (ems / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": ems, "steps": args.e2e_steps,
+               "entry_point": "adwin_opd_kl_fwd_bwd_host (pinned host logits in, host gradient out)",
+               "matches_device_path": same}
+
+    # ---- CPU oracle beside it (rank 0, one GPU only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        seqs = [b for b in range(B) if int(win_h[b]) >= 1024][:4] or [0]
+        nrows = 1024
+        sample = sample_rows_for_oracle(batch, seqs, nrows)
+        n, dt, cores = oracle_sample(sample)
+        cpu = {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"first {nrows} window rows of {len(seqs)} sequences of the same batch "
+                         f"({n} rows, {dt:.1f} s)"}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peak, peak_src = measured_peak()
+    alg_bytes = rows * V * 6            # per launch on one GPU: 2 reads + 1 write of bf16 per entry
+    achieved = alg_bytes / (kernel_ms * 1e-3) / 1e9
+    tr = recorded_traffic()
+    traffic = None
+    if tr and tr.get("rows"):
+        traffic = tr["dram_bytes"] * rows / tr["rows"]
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "storage_dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "in_window_rows_per_gpu": rows,
+                   "l2": "no flush needed: each step streams 14 GB, far larger than the 126 MB L2",
+                   "parallelism": f"dp{world} (independent batches per rank, no collective)"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                     "kernel": "kl_staged_kernel<bf16,bf16> (timed with the row-map kernel it "
+                               "follows, < 0.5 % of the interval)",
+                     "kernel_ms": kernel_ms, "algorithmic_bytes": alg_bytes,
+                     "frac_of_nominal_8TBps": achieved / 8000.0},
+        "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": LAUNCHES_PER_STEP * args.steps,
+        "clocks": clocks, "windowed_kl_sum": loss,
+        "L_next": int(al.L_next.item()),
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

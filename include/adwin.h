@@ -36,7 +36,7 @@ typedef enum {
   ADWIN_ERR_SHAPE = 2,       /* B, T, V, ld, K out of range */
   ADWIN_ERR_ALIGN = 3,       /* a pointer is not aligned to its element type */
   ADWIN_ERR_DTYPE = 4,       /* unknown dtype / grad mode / flag */
-  ADWIN_ERR_WINDOW = 5,      /* reserved for host-visible window errors */
+  ADWIN_ERR_WINDOW = 5,      /* a host-visible W_b or R_b is negative, or R_b > T */
   ADWIN_ERR_WORKSPACE = 6,   /* workspace NULL, misaligned or smaller than adwin_workspace_bytes */
   ADWIN_ERR_CUDA = 7,        /* a CUDA runtime call failed (launch, attribute, copy) */
   ADWIN_ERR_UNSUPPORTED = 8  /* the requested combination is not implemented */
@@ -157,6 +157,34 @@ int adwin_probe_align(const float* kl, const float* logratio, const float* gsq,
                       const int32_t* candidates, int32_t K, double rho_star, double* seq_stats,
                       double* seq_full, double* batch_stats, int32_t* L_next, int32_t* flags_out,
                       void* cuda_stream);
+
+/*
+ * The same pass for logits that live in HOST memory (pinned memory gives asynchronous copies).
+ * Only the rows inside the processed range cross PCIe -- the window skip of Section 4.1 saves the
+ * transfer as well as the arithmetic -- in stages of at most rows_per_stage rows of one sequence;
+ * copies in, kernels and read-backs of neighbouring stages overlap on three streams (the kernels
+ * run on cuda_stream; two internal copy streams are created on first use, per device).
+ *
+ * student_host, teacher_host, tokens_host, window_host, rollout_len_host, grad_host, kl_host,
+ * logratio_host, gsq_host: HOST pointers with the shapes / strides of adwin_opd_kl_fwd_bwd.
+ * The int32 length arrays are read during the call; everything else is read or written
+ * asynchronously: synchronise cuda_stream before touching the outputs or reusing the inputs.
+ * staging_dev : DEVICE scratch of >= adwin_host_staging_bytes(...) bytes, 256-byte aligned.
+ * dev_status  : DEVICE int32, as in adwin_opd_kl_fwd_bwd.
+ * Invalid lengths are host-visible here and return ADWIN_ERR_WINDOW before anything is enqueued.
+ * The paper has no counterpart for this entry point: it is the end-to-end form of Section 4.1's
+ * prefix evaluation for a trainer whose logits are produced on another device or host.
+ */
+size_t adwin_host_staging_bytes(int64_t rows_per_stage, int64_t V, int dtype, int grad_dtype,
+                                int with_grad);
+int adwin_opd_kl_fwd_bwd_host(const void* student_host, const void* teacher_host, int dtype,
+                              int64_t B, int64_t T, int64_t V, int64_t ld,
+                              const int32_t* tokens_host, const int32_t* window_host,
+                              const int32_t* rollout_len_host, float grad_scale, int grad_mode,
+                              int flags, void* grad_host, int grad_dtype, int64_t ld_grad,
+                              float* kl_host, float* logratio_host, float* gsq_host,
+                              void* staging_dev, size_t staging_bytes, int64_t rows_per_stage,
+                              int32_t* dev_status, void* cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -25,7 +25,8 @@ DEFAULT_CANDIDATES = (64, 128, 256, 512, 1024, 2048)   # Section 5.1, Training D
 RHO_STAR = math.sqrt(2.0) / 2.0                          # Eq. 5
 
 EXPORTS = ("adwin_version", "adwin_status_string", "adwin_workspace_bytes",
-           "adwin_opd_kl_fwd_bwd", "adwin_window_reduce", "adwin_probe_align")
+           "adwin_opd_kl_fwd_bwd", "adwin_window_reduce", "adwin_probe_align",
+           "adwin_host_staging_bytes", "adwin_opd_kl_fwd_bwd_host")
 
 _lib = None
 
@@ -61,6 +62,12 @@ def lib():
         L.adwin_probe_align.restype = ctypes.c_int
         L.adwin_probe_align.argtypes = [vp, vp, vp, vp, vp, i64, i64, vp, i32, f64, vp, vp, vp,
                                         vp, vp, vp]
+        L.adwin_host_staging_bytes.restype = sz
+        L.adwin_host_staging_bytes.argtypes = [i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_int]
+        L.adwin_opd_kl_fwd_bwd_host.restype = ctypes.c_int
+        L.adwin_opd_kl_fwd_bwd_host.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, i64, vp, vp,
+                                                vp, f32, ctypes.c_int, ctypes.c_int, vp,
+                                                ctypes.c_int, i64, vp, vp, vp, vp, sz, i64, vp, vp]
         _lib = L
     return _lib
 
@@ -180,4 +187,47 @@ def adwin_probe_align(kl, logratio, gsq, window, rollout_len=None, candidates=No
                                    _ptr(rollout_len), B, T, _ptr(candidates), K, float(rho_star),
                                    _ptr(o.seq_stats), _ptr(o.seq_full), _ptr(o.batch_stats),
                                    _ptr(o.L_next), _ptr(o.flags), _stream(dev)))
+    return o
+
+
+def adwin_host_staging_bytes(rows_per_stage, V, dtype, grad_dtype, with_grad=True) -> int:
+    return int(lib().adwin_host_staging_bytes(rows_per_stage, V, dtype, grad_dtype,
+                                              1 if with_grad else 0))
+
+
+def adwin_opd_kl_fwd_bwd_host(student, teacher, tokens, window, rollout_len=None, *, device,
+                              grad=None, grad_scale=1.0, grad_mode=GRAD_FULL_KL, flags=0,
+                              rows_per_stage=256, want_gsq=True, out=None, staging=None,
+                              dev_status=None):
+    """Host-buffer form: every tensor argument lives in (preferably pinned) host memory.
+
+    Returns a namespace with host tensors kl, logratio, gsq, grad and the device status word.
+    Asynchronous: synchronise the current stream of ``device`` before reading the outputs.
+    """
+    assert not student.is_cuda and not teacher.is_cuda and student.shape == teacher.shape
+    B, T, V = student.shape
+    assert student.is_contiguous() and teacher.is_contiguous()
+    dev = torch.device(device)
+    o = out if out is not None else SimpleNamespace()
+    if getattr(o, "kl", None) is None:
+        pin = dict(dtype=torch.float32, pin_memory=True)
+        o.kl = torch.empty((B, T), **pin)
+        o.logratio = torch.empty((B, T), **pin)
+        o.gsq = torch.empty((B, T), **pin) if want_gsq else None
+    o.grad = grad
+    dt = _dtype_code(student.dtype)
+    gdt = _dtype_code(grad.dtype) if grad is not None else dt
+    need = adwin_host_staging_bytes(rows_per_stage, V, dt, gdt, grad is not None)
+    if staging is None:
+        staging = torch.empty(need, dtype=torch.uint8, device=dev)
+    if dev_status is None:
+        dev_status = torch.zeros(1, dtype=torch.int32, device=dev)
+    o.dev_status, o.staging = dev_status, staging
+    with torch.cuda.device(dev):
+        rc = lib().adwin_opd_kl_fwd_bwd_host(
+            _ptr(student), _ptr(teacher), dt, B, T, V, V, _ptr(tokens), _ptr(window),
+            _ptr(rollout_len), float(grad_scale), int(grad_mode), int(flags), _ptr(grad), gdt, V,
+            _ptr(o.kl), _ptr(o.logratio), _ptr(o.gsq), _ptr(staging), staging.numel(),
+            int(rows_per_stage), _ptr(dev_status), _stream(dev))
+    _check(rc)
     return o

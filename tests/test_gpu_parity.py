@@ -255,3 +255,32 @@ def test_probe_align_default_candidates_and_flags():
     al = api.adwin_probe_align(kl, c, gsq1, win, None, rho_star=0.9)
     torch.cuda.synchronize()
     assert int(al.flags.item()) & api.ALIGN_NONE_ADMISSIBLE and int(al.L_next.item()) == 2048
+
+
+@pytest.mark.parametrize("flags", [0, api.RANGE_FULL | api.ZERO_TAIL])
+def test_host_buffer_entry_point_matches_device_entry_point(flags):
+    batch = synth.make_batch(2, device="cpu", B=3, T=70, V=8192, ragged_rollout=True)
+    batch.window = torch.tensor([70, 9, 33], dtype=torch.int32)
+    batch.rollout_len = torch.tensor([70, 40, 20], dtype=torch.int32)
+    pin = lambda x: x.contiguous().pin_memory()
+    s_h, t_h, tok_h = pin(batch.student), pin(batch.teacher), pin(batch.tokens)
+    g_h = torch.full(batch.shape, 5.0, dtype=torch.bfloat16).pin_memory()
+    got = api.adwin_opd_kl_fwd_bwd_host(s_h, t_h, tok_h, batch.window, batch.rollout_len,
+                                        device=DEV, grad=g_h, flags=flags, rows_per_stage=16,
+                                        grad_scale=0.5)
+    torch.cuda.synchronize()
+    assert int(got.dev_status.item()) == 0
+    dgrad = torch.full(batch.shape, 5.0, dtype=torch.bfloat16, device=DEV)
+    ref = api.adwin_opd_kl_fwd_bwd(batch.student.to(DEV), batch.teacher.to(DEV),
+                                   batch.tokens.to(DEV), batch.window.to(DEV),
+                                   batch.rollout_len.to(DEV), grad=dgrad, flags=flags,
+                                   grad_scale=0.5)
+    torch.cuda.synchronize()
+    # same kernels on the same values: only the staging layout differs
+    assert torch.allclose(got.kl, ref.kl.cpu(), rtol=1e-6, atol=1e-7)
+    assert torch.allclose(got.logratio, ref.logratio.cpu(), rtol=1e-6, atol=1e-7)
+    assert torch.allclose(got.gsq, ref.gsq.cpu(), rtol=1e-5, atol=1e-12)
+    assert torch.equal(g_h, dgrad.cpu())
+    with pytest.raises(api.AdwinError):
+        api.adwin_opd_kl_fwd_bwd_host(s_h, t_h, tok_h, torch.tensor([-1, 2, 3], dtype=torch.int32),
+                                      None, device=DEV)
