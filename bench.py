@@ -44,7 +44,9 @@ def parse():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--seqs", type=int, default=None, help="override B (debugging only)")
+    ap.add_argument("--seqs", type=int, default=None, help="override B (profiling a small case only)")
+    ap.add_argument("--positions", type=int, default=None,
+                    help="override T (profiling a small case only)")
     return ap.parse_args()
 
 
@@ -223,7 +225,8 @@ def run_ours(args):
     build.build()
     api.lib()
 
-    batch = synth.make_batch(3, device=dev, seed=synth.SEED_BASE + 100000 * rank, B=args.seqs)
+    batch = synth.make_batch(3, device=dev, seed=synth.SEED_BASE + 100000 * rank, B=args.seqs,
+                             T=args.positions)
     B, T, V = batch.shape
     win_h = torch.minimum(batch.window, batch.rollout_len).cpu()
     rows = int(win_h.sum())
