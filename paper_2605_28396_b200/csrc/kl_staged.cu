@@ -1,24 +1,37 @@
 // Staged cluster kernel: each logit byte is read from HBM once.
 //
 // A thread-block cluster of CL CTAs owns one processed row at a time; CTA `rank` owns a contiguous
-// slice of the vocabulary.  A producer warp streams the slice of z and of u into a shared-memory
-// ring with bulk asynchronous copies (cp.async.bulk, one mbarrier per ring slot); 16 consumer
-// warps make sweep 1 over the chunks as they land (online log-sum-exp of both rows, sum e*delta,
-// moments of the gradient norm), the CL partial results are exchanged through distributed shared
-// memory (remote stores + remote mbarrier arrive), and sweep 2 re-reads the slice from shared
-// memory -- not from HBM -- to write the gradient with 16-byte coalesced stores.  A slot is
-// handed back to the producer as soon as sweep 2 (or sweep 1, for rows whose gradient is not
-// written) has read it, so the next row's chunks stream in underneath the current row's compute.
-// Clusters are persistent and walk the compact list of in-window rows; rows past the window
-// cost nothing.
+// slice of the vocabulary.  Three kinds of warps share a CTA:
+//   * one producer warp streams the slice of z and of u into a shared-memory ring with bulk
+//     asynchronous copies (cp.async.bulk, one mbarrier per ring slot);
+//   * 16 consumer warps make sweep 1 over the chunks as they land (log-sum-exp statistics of both
+//     rows, sum e*delta, and for rows without a gradient the moments of its squared norm) and
+//     sweep 2, which re-reads the slice from shared memory -- not from HBM -- and writes the
+//     gradient with 16-byte coalesced stores;
+//   * one finisher warp combines the consumer warps' partial sums, exchanges the CTA's record
+//     with the CL-1 peers through distributed shared memory (remote stores + remote mbarrier
+//     arrive), derives the row's scalars and publishes them to the consumers.
+// When the ring holds two row slices (plan.lag == 1) the consumers run sweep 2 one row behind
+// sweep 1:  S1(i) -> S2(i-1) -> S1(i+1) -> ...  so the exchange of row i is hidden behind sweep 2
+// of row i-1 and no consumer warp ever waits for a peer CTA in steady state.  Otherwise
+// (plan.lag == 0) sweep 2 of a row follows its own sweep 1.  A slot goes back to the producer as
+// soon as its last reader is done with it, so the next rows' chunks stream in underneath the
+// current rows' arithmetic.  Clusters are persistent and walk the compact list of in-window rows;
+// rows past the window cost nothing.
 //
 // Ring invariant: chunks are numbered q = 0,1,2,... in the order rows are processed; chunk q lives
 // in slot q % nslot and is fill number q / nslot of that slot.  full[slot] completes once per fill
 // (producer arrive + transaction bytes), empty[slot] once per drain (one arrive per consumer warp).
+// Per-row hand-offs are double buffered by row parity: partready (consumers -> finisher, sweep-1
+// partials), rowready (finisher -> consumers, row scalars), qready (consumers -> finisher, squared
+// norm of the written gradient), xbar (peer finishers -> finisher, exchanged records).
 //
 // Every wait is bounded by a wall-clock limit; on expiry the CTA raises ADWIN_DEV_TIMEOUT, stops
 // waiting anywhere, drains its own copies, and still reaches the final cluster barrier so that no
 // peer is left behind.
+#include <mutex>
+#include <vector>
+
 #include "adwin_common.cuh"
 #include "adwin_internal.h"
 
@@ -26,7 +39,9 @@ namespace adwin {
 
 constexpr int kNT = 512;             // consumer threads
 constexpr int kNW = kNT / 32;        // consumer warps
-constexpr int kThreads = kNT + 32;   // + one producer warp
+constexpr int kProducerWarp = kNW;
+constexpr int kFinisherWarp = kNW + 1;
+constexpr int kThreads = kNT + 64;   // + producer warp + finisher warp
 constexpr int kMaxSlots = 32;
 constexpr int kMaxCL = 8;
 constexpr int kXF = 12;              // floats per exchange record
@@ -35,6 +50,7 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
 
 struct StagedPlan {
   int cl;                 // cluster size
+  int lag;                // 1: sweep 2 runs one row behind sweep 1 (two row slices resident)
   int nslot;              // ring slots
   int nch;                // chunks per slice (same for every rank)
   int chunk_pieces;       // 16-byte pieces per chunk (per array)
@@ -47,12 +63,15 @@ struct __align__(16) Ctrl {
   unsigned long long full[kMaxSlots];
   unsigned long long empty[kMaxSlots];
   unsigned long long xbar[2];
+  unsigned long long partready[2];
+  unsigned long long qready[2];
+  unsigned long long rowready[2];
   int abort_flag;
   int pad[3];
   float xbuf[2][kMaxCL][kXF];
-  float wpart[kNW][8];
-  float wq[kNW];
-  float rowres[16];
+  float wpart[2][kNW][8];
+  float wq[2][kNW];
+  float rowres[2][8];
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
@@ -131,12 +150,6 @@ __device__ __forceinline__ uint64_t global_timer() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-__device__ __forceinline__ void consumer_bar_sync(int id) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(kNT) : "memory");
-}
-__device__ __forceinline__ void consumer_bar_arrive(int id) {
-  asm volatile("bar.arrive %0, %1;" ::"r"(id), "n"(kNT) : "memory");
-}
 
 // Bounded wait.  Returns immediately (false) once the CTA has given up.
 template <bool CLUSTER>
@@ -173,7 +186,7 @@ __device__ __forceinline__ void load_piece(const char* slot, uint32_t u_off, int
 
 // ---------------------------------------------------------------------------- packed fp32 pairs
 // sm_100 issues add/mul/fma on two fp32 lanes held in a 64-bit register pair in one slot
-// (add.f32x2 / mul.f32x2 / fma.f32x2).  The sweeps are issue-bound, so all element-wise
+// (add.f32x2 / mul.f32x2 / fma.f32x2).  The sweeps are issue- and MUFU-bound, so all element-wise
 // arithmetic is done on pairs; only ex2 (MUFU) is per lane.
 typedef unsigned long long f2_t;
 
@@ -261,17 +274,17 @@ __device__ __forceinline__ void piece_max(const f2_t (&Z)[NP], const f2_t (&U)[N
 }
 
 // Rows whose gradient is written: fixed references (set from the thread's first piece), no
-// per-piece maximum.  The caller checks the sums for overflow after the sweep and, if a later
-// entry ran more than ~2^100 above the reference, redoes the slice with the online-maximum path
-// (the slice is still resident in shared memory).
+// per-piece maximum, delta = z - u uncentred.  The caller checks the sums for overflow after the
+// sweep and, if a later entry ran more than ~2^100 above the reference, redoes the slice with the
+// online-maximum path (the slice is still resident in shared memory).
 template <int NP>
 __device__ __forceinline__ void acc_fast(const f2_t (&Z)[NP], const f2_t (&U)[NP], f2_t nm2s,
-                                         f2_t nm2t, f2_t ndref, Acc2& a) {
+                                         f2_t nm2t, Acc2& a) {
   const f2_t L2 = splat2(kLog2e), NEG1 = splat2(-1.f);
 #pragma unroll
   for (int i = 0; i < NP; ++i) {
     const f2_t E = ex2_2(fma2(Z[i], L2, nm2s));
-    const f2_t D = add2(fma2(U[i], NEG1, Z[i]), ndref);
+    const f2_t D = fma2(U[i], NEG1, Z[i]);
     a.S = add2(a.S, E);
     a.A = fma2(E, D, a.A);
     a.St = add2(a.St, ex2_2(fma2(U[i], L2, nm2t)));
@@ -279,7 +292,7 @@ __device__ __forceinline__ void acc_fast(const f2_t (&Z)[NP], const f2_t (&U)[NP
 }
 
 // Rows whose gradient is not written (probe rows): online maximum per piece, plus the moments
-// sum e^2 {1, delta, delta^2} of the single-sweep squared gradient norm.
+// sum e^2 {1, delta, delta^2} of the single-sweep squared gradient norm, delta centred on dref.
 template <int NP>
 __device__ __forceinline__ void acc_probe(const f2_t (&Z)[NP], const f2_t (&U)[NP], float dref,
                                           Acc2& a) {
@@ -342,26 +355,28 @@ __device__ __forceinline__ void store_pairs(char* dst, const f2_t (&G)[NP]) {
   }
 }
 
-template <typename TOut, int N>
-__device__ __forceinline__ void store_piece(char* grow, int64_t piece_global, const float (&g)[N]) {
-  if (sizeof(TOut) == 4) {
-    float4* o = reinterpret_cast<float4*>(grow) + piece_global * (N / 4);
-#pragma unroll
-    for (int j = 0; j < N / 4; ++j)
-      __stcs(o + j, make_float4(g[4 * j], g[4 * j + 1], g[4 * j + 2], g[4 * j + 3]));
-  } else if (N == 8) {
-    uint4 o;
-    o.x = pack_bf16x2(g[0], g[1]);
-    o.y = pack_bf16x2(g[2], g[3]);
-    o.z = pack_bf16x2(g[4], g[5]);
-    o.w = pack_bf16x2(g[6], g[7]);
-    __stcs(reinterpret_cast<uint4*>(grow) + piece_global, o);
-  } else {
-    uint2 o;
-    o.x = pack_bf16x2(g[0], g[1]);
-    o.y = pack_bf16x2(g[2], g[3]);
-    __stcs(reinterpret_cast<uint2*>(grow) + piece_global, o);
+// Row metadata shared by the consumer and finisher roles: which global row, whether its gradient
+// is written, its sampled token and the two logits at that token.
+struct RowCursor {
+  int64_t b;   // monotone sequence pointer
+  __device__ __forceinline__ void fetch_row(const KlParams& p, int64_t ordinal, bool in_range,
+                                            int64_t& r, int& y, bool& wg) {
+    if (in_range) {
+      r = locate_row(p, ordinal, b);
+      const int64_t bb = r / p.T;
+      wg = (p.grad != nullptr) && ((r - bb * p.T) < p.ewin[bb]);
+      y = p.tokens[r];
+    }
   }
+};
+
+template <typename TIn>
+__device__ __forceinline__ void fetch_logits_at(const KlParams& p, int64_t r, int y, float& zy,
+                                                float& uy) {
+  const bool ok = (y >= 0) && ((int64_t)y < p.V);
+  const int64_t yi = ok ? y : 0;
+  zy = Elem<TIn>::load1(static_cast<const char*>(p.student) + (size_t)r * p.ld * sizeof(TIn), yi);
+  uy = Elem<TIn>::load1(static_cast<const char*>(p.teacher) + (size_t)r * p.ld * sizeof(TIn), yi);
 }
 
 template <typename TIn, typename TOut>
@@ -377,6 +392,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
   const int warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_rank();
   const int cl = plan.cl;
+  const int lag = plan.lag;
   const int64_t cluster_id = blockIdx.x / cl;
   const uint32_t u_off = (uint32_t)plan.chunk_pieces * 16u;
 
@@ -395,15 +411,25 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       mbar_init(smem_u32(&ctrl.full[s]), 1);
       mbar_init(smem_u32(&ctrl.empty[s]), kNW);
     }
-    mbar_init(smem_u32(&ctrl.xbar[0]), cl);
-    mbar_init(smem_u32(&ctrl.xbar[1]), cl);
+    for (int k = 0; k < 2; ++k) {
+      mbar_init(smem_u32(&ctrl.xbar[k]), cl);
+      mbar_init(smem_u32(&ctrl.partready[k]), kNW);
+      mbar_init(smem_u32(&ctrl.qready[k]), kNW);
+      mbar_init(smem_u32(&ctrl.rowready[k]), 1);
+    }
     ctrl.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
   cluster_sync_all();  // peers' barriers exist before any remote arrive
 
-  if (warp == kNW) {
+  // pieces of this CTA's slice that fall into chunk j (<= 0 for chunks past the slice end)
+  auto pieces_in_chunk = [&](int j) -> int {
+    const int left = (int)my_pieces - j * plan.chunk_pieces;
+    return left < plan.chunk_pieces ? left : plan.chunk_pieces;
+  };
+
+  if (warp == kProducerWarp) {
     // ------------------------------------------------------------------ producer warp
     if (lane == 0) {
       int slot = 0;
@@ -417,8 +443,8 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
         const char* urow = static_cast<const char*>(p.teacher) + ((size_t)r * p.ld + piece0 * N) * sizeof(TIn);
         for (int j = 0; j < plan.nch; ++j) {
           if (fills >= plan.nslot) bounded_wait<false>(smem_u32(&ctrl.empty[slot]), phase ^ 1u, abort);
-          int64_t np = my_pieces - (int64_t)j * plan.chunk_pieces;
-          np = np < 0 ? 0 : (np > plan.chunk_pieces ? plan.chunk_pieces : np);
+          int np = pieces_in_chunk(j);
+          np = np < 0 ? 0 : np;
           const uint32_t bytes = (uint32_t)np * 16u;
           const uint32_t bar = smem_u32(&ctrl.full[slot]);
           if (bytes == 0) {
@@ -455,79 +481,178 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       }
       if (gave_up) atomicOr(p.status, ADWIN_DEV_TIMEOUT);
     }
-  } else {
-    // ------------------------------------------------------------------ consumer warps
-    const bool full_mode = (p.mode == ADWIN_GRAD_FULL_KL);
-    int slot = 0;
-    uint32_t phase = 0;
-    bool timed_out = false;
-
-    // metadata pipeline: current row (C) and next row (N) held in registers
-    int64_t bptr = 0;
-    int64_t rC = 0, rN = 0;
+  } else if (warp == kFinisherWarp) {
+    // ------------------------------------------------------------------ finisher warp
+    // Iteration i < my_rows exchanges the sweep-1 record of row i; every iteration also carries the
+    // CTA's share of the squared gradient norm of row i-1-lag (written by sweep 2), so 1+lag
+    // trailing iterations deliver the last norms.  All CTAs of a cluster run the same iterations.
+    RowCursor cur;
+    cur.b = 0;
+    int64_t rC = 0, rN = 0, rH1 = 0, rH2 = 0;
     int yC = 0, yN = 0;
     float zyC = 0.f, uyC = 0.f;
-    bool wgC = false, wgN = false;
-    auto fetch_row = [&](int64_t i, int64_t& r, int& y, bool& wg) {
-      if (i < my_rows) {
-        r = locate_row(p, cluster_id + i * plan.num_clusters, bptr);
-        const int64_t bb = r / p.T;
-        wg = (p.grad != nullptr) && ((r - bb * p.T) < p.ewin[bb]);
-        y = p.tokens[r];
-      }
-    };
-    auto fetch_logits_at = [&](int64_t r, int y, float& zy, float& uy) {
-      const bool ok = (y >= 0) && ((int64_t)y < p.V);
-      const int64_t yi = ok ? y : 0;
-      zy = Elem<TIn>::load1(static_cast<const char*>(p.student) + (size_t)r * p.ld * sizeof(TIn), yi);
-      uy = Elem<TIn>::load1(static_cast<const char*>(p.teacher) + (size_t)r * p.ld * sizeof(TIn), yi);
-    };
-    fetch_row(0, rC, yC, wgC);
-    if (my_rows > 0) fetch_logits_at(rC, yC, zyC, uyC);
-    fetch_row(1, rN, yN, wgN);
-
-    int64_t pend_row = -1;   // row whose sweep-2 squared norm is still to be exchanged
-    float pend_q = 0.f;      // this thread's share of it (valid in lane 0 of each warp after reduce)
-
-    for (int64_t i = 0; i <= my_rows; ++i) {
-      const bool flush_only = (i == my_rows);   // one extra exchange delivers the last pending norm
-      if (flush_only && pend_row < 0) break;    // uniform across the cluster (same rows, same flags)
-
-      // issue next row's dependent loads early; they are consumed one row later
+    bool wgC = false, wgN = false, wgH1 = false, wgH2 = false;
+    cur.fetch_row(p, cluster_id, 0 < my_rows, rC, yC, wgC);
+    if (my_rows > 0) fetch_logits_at<TIn>(p, rC, yC, zyC, uyC);
+    cur.fetch_row(p, cluster_id + plan.num_clusters, 1 < my_rows, rN, yN, wgN);
+    bool timed_out = false;
+    const int64_t iters = my_rows > 0 ? my_rows + 1 + lag : 0;
+    for (int64_t i = 0; i < iters; ++i) {
+      const bool real = i < my_rows;
+      // next rows' dependent loads, consumed one iteration later
       float zyN = 0.f, uyN = 0.f;
       int64_t rNN = 0;
       int yNN = 0;
       bool wgNN = false;
-      if (!flush_only) {
-        if (i + 1 < my_rows) fetch_logits_at(rN, yN, zyN, uyN);
-        fetch_row(i + 2, rNN, yNN, wgNN);
+      if (i + 1 < my_rows) fetch_logits_at<TIn>(p, rN, yN, zyN, uyN);
+      cur.fetch_row(p, cluster_id + (i + 2) * plan.num_clusters, i + 2 < my_rows, rNN, yNN, wgNN);
+
+      const int par = (int)(i & 1);
+      const uint32_t ph = (uint32_t)((i >> 1) & 1);
+      float rec[8] = {-INFINITY, 0.f, 0.f, 0.f, 0.f, 0.f, -INFINITY, 0.f};
+      if (real) {
+        if (!bounded_wait<false>(smem_u32(&ctrl.partready[par]), ph, abort)) {
+          timed_out = true;
+          break;
+        }
+        // combine the consumer warps of this CTA (lane = source warp)
+        const bool has = lane < kNW;
+        const float* w = ctrl.wpart[par][has ? lane : 0];
+        const float ms = has ? w[0] : -INFINITY, mt = has ? w[6] : -INFINITY;
+        const float Ms = warp_max(ms), Mt = warp_max(mt);
+        const float fs = (ms == -INFINITY) ? 0.f : ex2f(ms - Ms);
+        const float ft = (mt == -INFINITY) ? 0.f : ex2f(mt - Mt);
+        const float fs2 = fs * fs;
+        rec[0] = Ms;
+        rec[1] = warp_sum(has ? w[1] * fs : 0.f);
+        rec[2] = warp_sum(has ? w[2] * fs : 0.f);
+        rec[3] = warp_sum(has ? w[3] * fs2 : 0.f);
+        rec[4] = warp_sum(has ? w[4] * fs2 : 0.f);
+        rec[5] = warp_sum(has ? w[5] * fs2 : 0.f);
+        rec[6] = Mt;
+        rec[7] = warp_sum(has ? w[7] * ft : 0.f);
       }
+      const int64_t jq = i - 1 - lag;               // row whose written-gradient norm is carried
+      const int64_t rq = lag ? rH2 : rH1;
+      const bool wgq = lag ? wgH2 : wgH1;
+      float qcta = 0.f;
+      if (jq >= 0) {
+        if (!bounded_wait<false>(smem_u32(&ctrl.qready[jq & 1]), (uint32_t)((jq >> 1) & 1), abort)) {
+          timed_out = true;
+          break;
+        }
+        qcta = warp_sum(lane < kNW ? ctrl.wq[jq & 1][lane] : 0.f);
+      }
+      // exchange: lane d delivers this CTA's record to peer d, then arrives on d's barrier
+      if (lane < cl) {
+        const uint32_t dst = map_to_rank(smem_u32(&ctrl.xbuf[par][rank][0]), (uint32_t)lane);
+        remote_store4(dst, rec[0], rec[1], rec[2], rec[3]);
+        remote_store4(dst + 16, rec[4], rec[5], rec[6], rec[7]);
+        remote_store4(dst + 32, qcta, 0.f, 0.f, 0.f);
+        remote_arrive_release(map_to_rank(smem_u32(&ctrl.xbar[par]), (uint32_t)lane));
+      }
+      if (!bounded_wait<true>(smem_u32(&ctrl.xbar[par]), ph, abort)) {
+        timed_out = true;
+        break;
+      }
+      // combine the CL records (lane = source rank); identical in every CTA of the cluster
+      RowTotals t;
+      float qtot;
+      {
+        const bool has = lane < cl;
+        const float* x = ctrl.xbuf[par][has ? lane : 0];
+        const float ms = has ? x[0] : -INFINITY, mt = has ? x[6] : -INFINITY;
+        t.M2s = warp_max(ms);
+        t.M2t = warp_max(mt);
+        const float fs = (ms == -INFINITY) ? 0.f : ex2f(ms - t.M2s);
+        const float ft = (mt == -INFINITY) ? 0.f : ex2f(mt - t.M2t);
+        const float fs2 = fs * fs;
+        t.S = warp_sum(has ? x[1] * fs : 0.f);
+        t.A = warp_sum(has ? x[2] * fs : 0.f);
+        t.B0 = warp_sum(has ? x[3] * fs2 : 0.f);
+        t.B1 = warp_sum(has ? x[4] * fs2 : 0.f);
+        t.B2 = warp_sum(has ? x[5] * fs2 : 0.f);
+        t.St = warp_sum(has ? x[7] * ft : 0.f);
+        qtot = warp_sum(has ? x[8] : 0.f);
+      }
+      if (lane == 0) {
+        if (rank == 0 && jq >= 0 && wgq && p.gsq) p.gsq[rq] = qtot;
+        if (real) {
+          const bool y_valid = (yC >= 0) && ((int64_t)yC < p.V);
+          const float dref = wgC ? 0.f : zyC - uyC;   // sweep 1 centres delta only on probe rows
+          const RowScalars rs = finish_row(t, zyC, uyC, y_valid, dref, p.alpha, p.mode);
+          float* rr = ctrl.rowres[par];
+          rr[0] = t.M2s;
+          rr[1] = rs.c0;
+          rr[2] = rs.coef;
+          rr[3] = rs.gy;
+          if (rank == 0) {
+            p.kl[rC] = rs.kl;
+            p.logratio[rC] = rs.c;
+            if (p.gsq && !wgC) p.gsq[rC] = rs.gsq_expanded;
+            if (p.lse_s) p.lse_s[rC] = rs.lse_s;
+            if (p.lse_t) p.lse_t[rC] = rs.lse_t;
+            int bits = 0;
+            if (!y_valid) bits |= ADWIN_DEV_TOKEN_RANGE;
+            if (rs.nonfinite) bits |= ADWIN_DEV_NONFINITE;
+            if (bits) atomicOr(p.status, bits);
+          }
+          mbar_arrive(smem_u32(&ctrl.rowready[par]));   // release: the row scalars are visible
+        }
+      }
+      __syncwarp();
+      // rotate the metadata pipeline
+      rH2 = rH1; wgH2 = wgH1;
+      rH1 = rC; wgH1 = wgC;
+      rC = rN; yC = yN; wgC = wgN; zyC = zyN; uyC = uyN;
+      rN = rNN; yN = yNN; wgN = wgNN;
+    }
+    if (timed_out && lane == 0) {
+      atomicOr(p.status, ADWIN_DEV_TIMEOUT);
+      for (int d = 0; d < cl; ++d)
+        remote_store_u32(map_to_rank(smem_u32(&ctrl.abort_flag), (uint32_t)d), 1u);
+    }
+  } else {
+    // ------------------------------------------------------------------ consumer warps
+    const bool full_mode = (p.mode == ADWIN_GRAD_FULL_KL);
+    int s1_slot = 0, s2_slot = 0;
+    uint32_t s1_phase = 0;
+    bool timed_out = false;
 
-      const bool y_valid = (yC >= 0) && ((int64_t)yC < p.V);
-      const float dref = zyC - uyC;
-      const int slot0 = slot;
-      // pieces of this CTA's slice that fall into chunk j (0 for chunks past the slice end)
-      auto pieces_in_chunk = [&](int j) -> int {
-        const int left = (int)my_pieces - j * plan.chunk_pieces;
-        return left < plan.chunk_pieces ? left : plan.chunk_pieces;
-      };
-      Acc2 a;
-      a.reset();
-      const int tpiece = tid;                      // this thread's piece inside every chunk
-      const uint32_t toff = (uint32_t)tid * 16u;
+    // metadata pipeline: row of this iteration's sweep 1 (C), the next one (N), the previous (P)
+    RowCursor cur;
+    cur.b = 0;
+    int64_t rC = 0, rN = 0, rP = 0;
+    int yC = 0, yN = 0, yP = 0;
+    float zyC = 0.f, uyC = 0.f;
+    bool wgC = false, wgN = false, wgP = false;
+    cur.fetch_row(p, cluster_id, 0 < my_rows, rC, yC, wgC);
+    if (my_rows > 0) fetch_logits_at<TIn>(p, rC, yC, zyC, uyC);
+    cur.fetch_row(p, cluster_id + plan.num_clusters, 1 < my_rows, rN, yN, wgN);
 
-      // ---------------------------------------------------------------- sweep 1
-      if (!flush_only) {
+    const uint32_t toff = (uint32_t)tid * 16u;   // this thread's piece inside every chunk
+    const int64_t iters = my_rows > 0 ? my_rows + lag : 0;
+    for (int64_t i = 0; i < iters; ++i) {
+      float zyN = 0.f, uyN = 0.f;
+      int64_t rNN = 0;
+      int yNN = 0;
+      bool wgNN = false;
+      if (i + 1 < my_rows) fetch_logits_at<TIn>(p, rN, yN, zyN, uyN);
+      cur.fetch_row(p, cluster_id + (i + 2) * plan.num_clusters, i + 2 < my_rows, rNN, yNN, wgNN);
+
+      // ---------------------------------------------------------------- sweep 1 of row i
+      if (i < my_rows) {
+        Acc2 a;
+        a.reset();
+        const int slot0 = s1_slot;
         if (wgC) {
           // gradient row: fixed references from the first piece, checked once after the sweep
           f2_t nm2s = 0ull, nm2t = 0ull;
-          const f2_t ndref = splat2(-dref);
           bool have_ref = false;
           for (int j = 0; j < plan.nch; ++j) {
-            if (!bounded_wait<false>(smem_u32(&ctrl.full[slot]), phase, abort)) timed_out = true;
-            const int np = pieces_in_chunk(j);
-            if (tpiece < np) {
-              const char* sl = ring + (size_t)slot * plan.slot_bytes + toff;
+            if (!bounded_wait<false>(smem_u32(&ctrl.full[s1_slot]), s1_phase, abort)) timed_out = true;
+            if (tid < pieces_in_chunk(j)) {
+              const char* sl = ring + (size_t)s1_slot * plan.slot_bytes + toff;
               f2_t Z[NP], U[NP];
               Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl), Z);
               Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl + u_off), U);
@@ -540,11 +665,11 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
                 nm2t = splat2(-a.m2t);
                 have_ref = true;
               }
-              acc_fast<NP>(Z, U, nm2s, nm2t, ndref, a);
+              acc_fast<NP>(Z, U, nm2s, nm2t, a);
             }
-            if (++slot == plan.nslot) {
-              slot = 0;
-              phase ^= 1u;
+            if (++s1_slot == plan.nslot) {
+              s1_slot = 0;
+              s1_phase ^= 1u;
             }
           }
           // overflow / invalid reference: redo this thread's pieces with the online maximum
@@ -552,15 +677,14 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
           if (!(hsum2(a.S) < kSumLimit) || !(hsum2(a.St) < kSumLimit)) {
             RowAcc ra;
             ra.reset();
-            int s2 = slot0;
+            int s = slot0;
             for (int j = 0; j < plan.nch; ++j) {
-              const int np = pieces_in_chunk(j);
-              if (tpiece < np) {
+              if (tid < pieces_in_chunk(j)) {
                 float z[N], u[N];
-                load_piece<TIn>(ring + (size_t)s2 * plan.slot_bytes, u_off, tpiece, z, u);
-                acc_piece<N, false>(z, u, dref, ra);
+                load_piece<TIn>(ring + (size_t)s * plan.slot_bytes, u_off, tid, z, u);
+                acc_piece<N, false>(z, u, 0.f, ra);
               }
-              if (++s2 == plan.nslot) s2 = 0;
+              if (++s == plan.nslot) s = 0;
             }
             a.reset();
             a.m2s = ra.m2s;
@@ -571,29 +695,26 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
           }
         } else {
           // probe row: nothing re-reads a chunk, so each slot goes back to the producer at once
+          const float dref = zyC - uyC;
           for (int j = 0; j < plan.nch; ++j) {
-            if (!bounded_wait<false>(smem_u32(&ctrl.full[slot]), phase, abort)) timed_out = true;
-            const int np = pieces_in_chunk(j);
-            if (tpiece < np) {
-              const char* sl = ring + (size_t)slot * plan.slot_bytes + toff;
+            if (!bounded_wait<false>(smem_u32(&ctrl.full[s1_slot]), s1_phase, abort)) timed_out = true;
+            if (tid < pieces_in_chunk(j)) {
+              const char* sl = ring + (size_t)s1_slot * plan.slot_bytes + toff;
               f2_t Z[NP], U[NP];
               Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl), Z);
               Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl + u_off), U);
               acc_probe<NP>(Z, U, dref, a);
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctrl.empty[slot]));
-            if (++slot == plan.nslot) {
-              slot = 0;
-              phase ^= 1u;
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl.empty[s1_slot]));
+            if (++s1_slot == plan.nslot) {
+              s1_slot = 0;
+              s1_phase ^= 1u;
             }
           }
         }
-      }
-
-
-      // ---------------------------------------------------------------- CTA reduction
-      {
+        if (timed_out) break;
+        // warp partials -> finisher
         const float wms = warp_max(a.m2s), wmt = warp_max(a.m2t);
         const float fs = (a.m2s == -INFINITY) ? 0.f : ex2f(a.m2s - wms);
         const float ft = (a.m2t == -INFINITY) ? 0.f : ex2f(a.m2t - wmt);
@@ -602,157 +723,85 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
         const float v2 = warp_sum(hsum2(a.B0) * fs2), v3 = warp_sum(hsum2(a.B1) * fs2);
         const float v4 = warp_sum(hsum2(a.B2) * fs2), v5 = warp_sum(hsum2(a.St) * ft);
         if (lane == 0) {
-          float* w = ctrl.wpart[warp];
+          float* w = ctrl.wpart[i & 1][warp];
           w[0] = wms; w[1] = v0; w[2] = v1; w[3] = v2; w[4] = v3; w[5] = v4; w[6] = wmt; w[7] = v5;
+          mbar_arrive(smem_u32(&ctrl.partready[i & 1]));
         }
       }
-      if (warp != 0) {
-        __threadfence_block();
-        consumer_bar_arrive(1);
-      } else {
-        consumer_bar_sync(1);
-        // warp 0: combine the warps of this CTA (lane = source warp)
-        float rec[8];
-        {
-          const bool has = lane < kNW;
-          const float* w = ctrl.wpart[has ? lane : 0];
-          const float ms = has ? w[0] : -INFINITY, mt = has ? w[6] : -INFINITY;
-          const float Ms = warp_max(ms), Mt = warp_max(mt);
-          const float fs = (ms == -INFINITY) ? 0.f : ex2f(ms - Ms);
-          const float ft = (mt == -INFINITY) ? 0.f : ex2f(mt - Mt);
-          const float fs2 = fs * fs;
-          rec[0] = Ms;
-          rec[1] = warp_sum(has ? w[1] * fs : 0.f);
-          rec[2] = warp_sum(has ? w[2] * fs : 0.f);
-          rec[3] = warp_sum(has ? w[3] * fs2 : 0.f);
-          rec[4] = warp_sum(has ? w[4] * fs2 : 0.f);
-          rec[5] = warp_sum(has ? w[5] * fs2 : 0.f);
-          rec[6] = Mt;
-          rec[7] = warp_sum(has ? w[7] * ft : 0.f);
-        }
-        const float qcta = warp_sum((lane < kNW && pend_row >= 0) ? ctrl.wq[lane] : 0.f);
-        // exchange: lane d delivers this CTA's record to peer d, then arrives on d's barrier
-        const int par = (int)(i & 1);
-        const uint32_t xphase = (uint32_t)((i >> 1) & 1);
-        if (lane < cl) {
-          const uint32_t dst = map_to_rank(smem_u32(&ctrl.xbuf[par][rank][0]), (uint32_t)lane);
-          remote_store4(dst, rec[0], rec[1], rec[2], rec[3]);
-          remote_store4(dst + 16, rec[4], rec[5], rec[6], rec[7]);
-          remote_store4(dst + 32, qcta, 0.f, 0.f, 0.f);
-          remote_arrive_release(map_to_rank(smem_u32(&ctrl.xbar[par]), (uint32_t)lane));
-        }
-        if (!bounded_wait<true>(smem_u32(&ctrl.xbar[par]), xphase, abort)) timed_out = true;
-        // combine the CL records (lane = source rank); identical in every CTA of the cluster
-        RowTotals t;
-        float qtot;
-        {
-          const bool has = lane < cl;
-          const float* x = ctrl.xbuf[par][has ? lane : 0];
-          const float ms = has ? x[0] : -INFINITY, mt = has ? x[6] : -INFINITY;
-          t.M2s = warp_max(ms);
-          t.M2t = warp_max(mt);
-          const float fs = (ms == -INFINITY) ? 0.f : ex2f(ms - t.M2s);
-          const float ft = (mt == -INFINITY) ? 0.f : ex2f(mt - t.M2t);
-          const float fs2 = fs * fs;
-          t.S = warp_sum(has ? x[1] * fs : 0.f);
-          t.A = warp_sum(has ? x[2] * fs : 0.f);
-          t.B0 = warp_sum(has ? x[3] * fs2 : 0.f);
-          t.B1 = warp_sum(has ? x[4] * fs2 : 0.f);
-          t.B2 = warp_sum(has ? x[5] * fs2 : 0.f);
-          t.St = warp_sum(has ? x[7] * ft : 0.f);
-          qtot = warp_sum(has ? x[8] : 0.f);
-        }
-        if (lane == 0) {
-          ctrl.rowres[4] = (*abort) ? 1.f : 0.f;   // one reader decides for the whole CTA
-          if (rank == 0 && pend_row >= 0 && p.gsq) p.gsq[pend_row] = qtot;
-          if (!flush_only) {
-            const RowScalars rs = finish_row(t, zyC, uyC, y_valid, dref, p.alpha, p.mode);
-            ctrl.rowres[0] = t.M2s;
-            ctrl.rowres[1] = rs.c0;
-            ctrl.rowres[2] = rs.coef;
-            ctrl.rowres[3] = rs.gy;
-            if (rank == 0) {
-              p.kl[rC] = rs.kl;
-              p.logratio[rC] = rs.c;
-              if (p.gsq && !wgC) p.gsq[rC] = rs.gsq_expanded;
-              if (p.lse_s) p.lse_s[rC] = rs.lse_s;
-              if (p.lse_t) p.lse_t[rC] = rs.lse_t;
-              int bits = 0;
-              if (!y_valid) bits |= ADWIN_DEV_TOKEN_RANGE;
-              if (rs.nonfinite) bits |= ADWIN_DEV_NONFINITE;
-              if (bits) atomicOr(p.status, bits);
-            }
-          }
-        }
-      }
-      consumer_bar_sync(2);   // row results (and the abort flag) are visible to every consumer
-      pend_row = -1;
-      if (ctrl.rowres[4] != 0.f) {
-        timed_out = true;
-        break;
-      }
-      if (flush_only) break;
 
-      // ---------------------------------------------------------------- sweep 2
-      if (wgC) {
-        const float M2s = ctrl.rowres[0], c0 = ctrl.rowres[1], coef = ctrl.rowres[2],
-                    gy = ctrl.rowres[3];
-        const f2_t L2 = splat2(kLog2e), NEG1 = splat2(-1.f);
-        const f2_t nM2s = splat2(-M2s), ndref = splat2(-dref), nc0 = splat2(-c0),
-                   coef2 = splat2(coef);
-        const int64_t ypiece = y_valid ? ((int64_t)yC / N - piece0) : -1;   // slice-relative
-        char* gthread = static_cast<char*>(p.grad) +
-                        ((size_t)rC * p.ld_grad + (size_t)(piece0 + tpiece) * N) * sizeof(TOut);
-        const size_t gstep = (size_t)plan.chunk_pieces * N * sizeof(TOut);
-        f2_t Q = 0ull;
-        int s2 = slot0;
-        for (int j = 0; j < plan.nch; ++j) {
-          const int np = pieces_in_chunk(j);
-          if (tpiece < np) {
-            const char* sl = ring + (size_t)s2 * plan.slot_bytes + toff;
-            f2_t Z[NP], U[NP], G[NP];
-            Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl), Z);
-            Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl + u_off), U);
-#pragma unroll
-            for (int k = 0; k < NP; ++k) {
-              const f2_t E = ex2_2(fma2(Z[k], L2, nM2s));
-              if (full_mode) {
-                const f2_t D = add2(add2(fma2(U[k], NEG1, Z[k]), ndref), nc0);
-                G[k] = mul2(E, mul2(D, coef2));
-              } else {
-                G[k] = mul2(E, coef2);
-              }
-            }
-            if (!full_mode && (int64_t)j * plan.chunk_pieces + tpiece == ypiece) {
-              const int e = (int)((int64_t)yC - ((int64_t)yC / N) * N);
+      // ---------------------------------------------------------------- sweep 2 of row i - lag
+      const int64_t j2 = i - lag;
+      if (j2 >= 0) {
+        const int64_t r2 = lag ? rP : rC;
+        const int y2 = lag ? yP : yC;
+        const bool wg2 = lag ? wgP : wgC;
+        const int par = (int)(j2 & 1);
+        if (!bounded_wait<false>(smem_u32(&ctrl.rowready[par]), (uint32_t)((j2 >> 1) & 1), abort)) {
+          timed_out = true;
+          break;
+        }
+        float q = 0.f;
+        if (wg2) {
+          const float M2s = ctrl.rowres[par][0], c0 = ctrl.rowres[par][1], coef = ctrl.rowres[par][2],
+                      gy = ctrl.rowres[par][3];
+          const bool y_valid = (y2 >= 0) && ((int64_t)y2 < p.V);
+          const f2_t L2 = splat2(kLog2e), NEG1 = splat2(-1.f);
+          const f2_t nM2s = splat2(-M2s), nc0 = splat2(-c0), coef2 = splat2(coef);
+          const int64_t ypiece = y_valid ? ((int64_t)y2 / N - piece0) : -1;   // slice-relative
+          char* gthread = static_cast<char*>(p.grad) +
+                          ((size_t)r2 * p.ld_grad + (size_t)(piece0 + tid) * N) * sizeof(TOut);
+          const size_t gstep = (size_t)plan.chunk_pieces * N * sizeof(TOut);
+          f2_t Q = 0ull;
+          for (int j = 0; j < plan.nch; ++j) {
+            if (tid < pieces_in_chunk(j)) {
+              const char* sl = ring + (size_t)s2_slot * plan.slot_bytes + toff;
+              f2_t Z[NP], U[NP], G[NP];
+              Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl), Z);
+              Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl + u_off), U);
 #pragma unroll
               for (int k = 0; k < NP; ++k) {
-                float lo, hi;
-                upk2(G[k], lo, hi);
-                if (e == 2 * k) lo = gy;
-                if (e == 2 * k + 1) hi = gy;
-                G[k] = pk2(lo, hi);
+                const f2_t E = ex2_2(fma2(Z[k], L2, nM2s));
+                if (full_mode) {
+                  const f2_t D = add2(fma2(U[k], NEG1, Z[k]), nc0);
+                  G[k] = mul2(E, mul2(D, coef2));
+                } else {
+                  G[k] = mul2(E, coef2);
+                }
               }
-            }
+              if (!full_mode && (int64_t)j * plan.chunk_pieces + tid == ypiece) {
+                const int e = (int)((int64_t)y2 - ((int64_t)y2 / N) * N);
 #pragma unroll
-            for (int k = 0; k < NP; ++k) Q = fma2(G[k], G[k], Q);
-            store_pairs<TOut, NP>(gthread + (size_t)j * gstep, G);
+                for (int k = 0; k < NP; ++k) {
+                  float lo, hi;
+                  upk2(G[k], lo, hi);
+                  if (e == 2 * k) lo = gy;
+                  if (e == 2 * k + 1) hi = gy;
+                  G[k] = pk2(lo, hi);
+                }
+              }
+#pragma unroll
+              for (int k = 0; k < NP; ++k) Q = fma2(G[k], G[k], Q);
+              store_pairs<TOut, NP>(gthread + (size_t)j * gstep, G);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl.empty[s2_slot]));
+            if (++s2_slot == plan.nslot) s2_slot = 0;
           }
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&ctrl.empty[s2]));
-          if (++s2 == plan.nslot) s2 = 0;
+          q = warp_sum(hsum2(Q));
+        } else {
+          s2_slot = (s2_slot + plan.nch) % plan.nslot;   // released by sweep 1 already
         }
-        const float q = warp_sum(hsum2(Q));
-        if (lane == 0) ctrl.wq[warp] = q;   // ordered before its use by the next row's bar 1
-        pend_row = rC;
-        pend_q = q;
+        if (lane == 0) {
+          ctrl.wq[par][warp] = q;
+          mbar_arrive(smem_u32(&ctrl.qready[par]));
+        }
       }
 
       // rotate the metadata pipeline
+      rP = rC; yP = yC; wgP = wgC;
       rC = rN; yC = yN; wgC = wgN; zyC = zyN; uyC = uyN;
       rN = rNN; yN = yNN; wgN = wgNN;
     }
-    (void)pend_q;
     if (timed_out && lane == 0) {
       atomicOr(p.status, ADWIN_DEV_TIMEOUT);
       // let the peers stop waiting as well
@@ -770,45 +819,136 @@ namespace {
 
 constexpr int kSmemOptin = 232448;   // 227 KB: the per-CTA limit of sm_100
 
-bool make_plan(const KlParams& p, int dtype, bool has_grad, StagedPlan& plan) {
-  const int N = dtype == ADWIN_F32 ? 4 : 8;
-  const int64_t pieces_total = p.V / N;
-  if (pieces_total < 1) return false;
+// Chunking of one cluster size; false when the slice does not fit the ring.
+bool plan_for_cluster(int64_t pieces_total, int cl, bool has_grad, StagedPlan& plan) {
   const int64_t ring_bytes = kSmemOptin - kCtrlBytes;
-  for (int cl = 1; cl <= kMaxCL; cl *= 2) {
-    const int64_t per_rank = (pieces_total + cl - 1) / cl;
-    int64_t nch, chunk_pieces;
-    if (has_grad) {
-      nch = (per_rank + kNT - 1) / kNT;
-      chunk_pieces = (per_rank + nch - 1) / nch;
-    } else {
-      chunk_pieces = per_rank < kNT ? per_rank : kNT;
-      nch = (per_rank + chunk_pieces - 1) / chunk_pieces;
-    }
-    const int64_t slot_bytes = 2 * chunk_pieces * 16;
-    int64_t nslot = ring_bytes / slot_bytes;
-    if (nslot > kMaxSlots) nslot = kMaxSlots;
-    const bool fits = has_grad ? (nch + 2 <= nslot) : (nslot >= 2);
-    if (!fits) continue;
-    if (per_rank * N * (dtype == ADWIN_F32 ? 4 : 2) > (int64_t)1 << 30) return false;
-    plan.cl = cl;
-    plan.nslot = (int)nslot;
-    plan.nch = (int)nch;
-    plan.chunk_pieces = (int)chunk_pieces;
-    plan.per_rank_pieces = (int)per_rank;
-    plan.slot_bytes = (uint32_t)slot_bytes;
-    return true;
+  const int64_t per_rank = (pieces_total + cl - 1) / cl;
+  if (per_rank * 16 > (int64_t)1 << 30) return false;
+  int64_t nch, chunk_pieces;
+  if (has_grad) {
+    nch = (per_rank + kNT - 1) / kNT;
+    chunk_pieces = (per_rank + nch - 1) / nch;
+  } else {
+    chunk_pieces = per_rank < kNT ? per_rank : kNT;
+    nch = (per_rank + chunk_pieces - 1) / chunk_pieces;
   }
-  return false;
+  chunk_pieces = (chunk_pieces + 7) / 8 * 8;   // slots start on 128-byte boundaries
+  if (chunk_pieces > kNT) chunk_pieces = kNT;
+  nch = (per_rank + chunk_pieces - 1) / chunk_pieces;
+  const int64_t slot_bytes = 2 * chunk_pieces * 16;
+  int64_t nslot = ring_bytes / slot_bytes;
+  if (nslot > kMaxSlots) nslot = kMaxSlots;
+  int lag = 0;
+  if (has_grad) {
+    if (2 * nch + 1 <= nslot) lag = 1;          // two row slices resident + one slot in flight
+    else if (nch + 2 > nslot) return false;     // one row slice + two slots in flight
+  } else {
+    if (nslot < 2) return false;
+    lag = 1;   // no slot is held for a second sweep: only the wait for the row scalars is deferred
+  }
+  plan.cl = cl;
+  plan.lag = lag;
+  plan.nslot = (int)nslot;
+  plan.nch = (int)nch;
+  plan.chunk_pieces = (int)chunk_pieces;
+  plan.per_rank_pieces = (int)per_rank;
+  plan.slot_bytes = (uint32_t)slot_bytes;
+  return true;
 }
 
 template <typename TIn, typename TOut>
-cudaError_t launch_staged_t(const KlParams& p, StagedPlan plan, int sm_count, cudaStream_t s) {
+cudaError_t max_clusters_for(const StagedPlan& plan, int sm_count, int& max_clusters) {
   auto kernel = kl_staged_kernel<TIn, TOut>;
   const int smem = kCtrlBytes + plan.nslot * (int)plan.slot_bytes;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = plan.cl;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cfg.gridDim = dim3(plan.cl * sm_count);
+  return cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg);
+}
 
+// The cluster size is chosen once per (device, shape class): among the sizes whose slice fits,
+// prefer plans that hide the exchange (lag 1), then the one that keeps the most SMs busy (cluster
+// sizes that do not divide a GPC's SM count leave SMs idle), then the smaller cluster.
+struct PlanKey {
+  int dev, dtype, grad_dtype, has_grad;
+  int64_t pieces_total;
+  bool operator==(const PlanKey& o) const {
+    return dev == o.dev && dtype == o.dtype && grad_dtype == o.grad_dtype &&
+           has_grad == o.has_grad && pieces_total == o.pieces_total;
+  }
+};
+struct PlanEntry {
+  PlanKey key;
+  bool ok;
+  StagedPlan plan;
+};
+
+template <typename TIn, typename TOut>
+bool choose_plan(int64_t pieces_total, bool has_grad, int sm_count, StagedPlan& best) {
+  double best_score = -1.0;
+  for (int cl = 1; cl <= kMaxCL; ++cl) {
+    StagedPlan plan = {};
+    if (!plan_for_cluster(pieces_total, cl, has_grad, plan)) continue;
+    int clusters = 0;
+    if (max_clusters_for<TIn, TOut>(plan, sm_count, clusters) != cudaSuccess) {
+      cudaGetLastError();
+      continue;
+    }
+    if (clusters < 1) continue;
+    const double ctas = (double)clusters * cl;
+    const double score = ctas * ((plan.lag || !has_grad) ? 1.0 : 0.6) - 1e-3 * cl;
+    if (score > best_score) {
+      best_score = score;
+      best = plan;
+      best.num_clusters = clusters;
+    }
+  }
+  return best_score > 0.0;
+}
+
+template <typename TIn, typename TOut>
+cudaError_t launch_staged_t(const KlParams& p, int dtype, int grad_dtype, int sm_count,
+                            cudaStream_t s) {
+  static std::mutex mu;
+  static std::vector<PlanEntry> cache;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const int N = dtype == ADWIN_F32 ? 4 : 8;
+  const PlanKey key = {dev, dtype, grad_dtype, p.grad != nullptr ? 1 : 0, p.V / N};
+  if (key.pieces_total < 1) return cudaErrorNotSupported;
+  StagedPlan plan = {};
+  bool ok = false, found = false;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    for (const PlanEntry& c : cache)
+      if (c.key == key) {
+        plan = c.plan;
+        ok = c.ok;
+        found = true;
+        break;
+      }
+    if (!found) {
+      ok = choose_plan<TIn, TOut>(key.pieces_total, key.has_grad != 0, sm_count, plan);
+      cache.push_back({key, ok, plan});
+    }
+  }
+  if (!ok) return cudaErrorNotSupported;
+
+  auto kernel = kl_staged_kernel<TIn, TOut>;
+  const int smem = kCtrlBytes + plan.nslot * (int)plan.slot_bytes;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = (size_t)smem;
@@ -820,16 +960,9 @@ cudaError_t launch_staged_t(const KlParams& p, StagedPlan plan, int sm_count, cu
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-
-  int max_clusters = 0;
-  cfg.gridDim = dim3(plan.cl * sm_count);
-  e = cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg);
-  if (e != cudaSuccess) return e;
-  if (max_clusters < 1) return cudaErrorNotSupported;
   const int64_t rows = p.B * p.T;
-  if (max_clusters > rows) max_clusters = (int)rows;
-  plan.num_clusters = max_clusters;
-  cfg.gridDim = dim3(plan.cl * max_clusters);
+  if (plan.num_clusters > rows) plan.num_clusters = (int)rows;
+  cfg.gridDim = dim3(plan.cl * plan.num_clusters);
   return cudaLaunchKernelEx(&cfg, kernel, p, plan);
 }
 
@@ -837,14 +970,14 @@ cudaError_t launch_staged_t(const KlParams& p, StagedPlan plan, int sm_count, cu
 
 cudaError_t launch_kl_staged(const KlParams& p, int dtype, int grad_dtype, int sm_count,
                              cudaStream_t s) {
-  StagedPlan plan = {};
-  if (!make_plan(p, dtype, p.grad != nullptr, plan)) return cudaErrorNotSupported;
   if (dtype == ADWIN_F32) {
-    return grad_dtype == ADWIN_F32 ? launch_staged_t<float, float>(p, plan, sm_count, s)
-                                   : launch_staged_t<float, __nv_bfloat16>(p, plan, sm_count, s);
+    return grad_dtype == ADWIN_F32
+               ? launch_staged_t<float, float>(p, dtype, grad_dtype, sm_count, s)
+               : launch_staged_t<float, __nv_bfloat16>(p, dtype, grad_dtype, sm_count, s);
   }
-  return grad_dtype == ADWIN_F32 ? launch_staged_t<__nv_bfloat16, float>(p, plan, sm_count, s)
-                                 : launch_staged_t<__nv_bfloat16, __nv_bfloat16>(p, plan, sm_count, s);
+  return grad_dtype == ADWIN_F32
+             ? launch_staged_t<__nv_bfloat16, float>(p, dtype, grad_dtype, sm_count, s)
+             : launch_staged_t<__nv_bfloat16, __nv_bfloat16>(p, dtype, grad_dtype, sm_count, s);
 }
 
 }  // namespace adwin
