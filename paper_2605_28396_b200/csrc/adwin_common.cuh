@@ -167,7 +167,8 @@ struct RowScalars {
 
 // Finalise one row from its totals (fp32; cheap enough for every thread to evaluate).
 // zy, uy: logits at the sampled token (ignored when !y_valid); dref as used in the sweep.
-//   lse = (M2 + log2 S) ln 2;  Delta = lse_s - lse_t;  E_p[delta] = A/S + dref
+//   lse = (M2 + log2 S) ln 2;  Delta = lse_s - lse_t = ((M2s - M2t) + log2(S/St)) ln 2;
+//   E_p[delta] = A/S + dref
 //   KL = E_p[delta] - Delta;   c = (z_y - u_y) - Delta
 // The expanded squared norm sum p^2 (delta - E_p delta)^2 = (B2 - 2 c0 B1 + c0^2 B0) / S^2 is only
 // used for rows whose gradient is not written.
@@ -178,7 +179,9 @@ __device__ __forceinline__ RowScalars finish_row(const RowTotals& t, float zy, f
   const float l2s = log2f(t.S), l2t = log2f(t.St);
   r.lse_s = (t.M2s + l2s) * kLn2f;
   r.lse_t = (t.M2t + l2t) * kLn2f;
-  const float delta = ((t.M2s - t.M2t) + (l2s - l2t)) * kLn2f;
+  // log2 S - log2 St as one logarithm of the ratio: both sums can be large against a shared
+  // reference, and their separate logarithms would each carry an absolute error of an ulp of ~20.
+  const float delta = ((t.M2s - t.M2t) + log2f(t.S / t.St)) * kLn2f;
   const float inv_s = 1.f / t.S;
   r.c0 = t.A * inv_s;
   r.kl = (r.c0 + dref) - delta;

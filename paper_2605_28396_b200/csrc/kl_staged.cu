@@ -1,34 +1,38 @@
 // Staged cluster kernel: each logit byte is read from HBM once.
 //
-// A thread-block cluster of CL CTAs owns one processed row at a time; CTA `rank` owns a contiguous
-// slice of the vocabulary.  Three kinds of warps share a CTA:
-//   * one producer warp streams the slice of z and of u into a shared-memory ring with bulk
-//     asynchronous copies (cp.async.bulk, one mbarrier per ring slot);
-//   * 16 consumer warps make sweep 1 over the chunks as they land (log-sum-exp statistics of both
-//     rows, sum e*delta, and for rows without a gradient the moments of its squared norm) and
-//     sweep 2, which re-reads the slice from shared memory -- not from HBM -- and writes the
-//     gradient with 16-byte coalesced stores;
-//   * one finisher warp combines the consumer warps' partial sums, exchanges the CTA's record
-//     with the CL-1 peers through distributed shared memory (remote stores + remote mbarrier
-//     arrive), derives the row's scalars and publishes them to the consumers.
-// When the ring holds two row slices (plan.lag == 1) the consumers run sweep 2 one row behind
-// sweep 1:  S1(i) -> S2(i-1) -> S1(i+1) -> ...  so the exchange of row i is hidden behind sweep 2
-// of row i-1 and no consumer warp ever waits for a peer CTA in steady state.  Otherwise
-// (plan.lag == 0) sweep 2 of a row follows its own sweep 1.  A slot goes back to the producer as
-// soon as its last reader is done with it, so the next rows' chunks stream in underneath the
-// current rows' arithmetic.  Clusters are persistent and walk the compact list of in-window rows;
-// rows past the window cost nothing.
+// A thread-block cluster of CL CTAs (one CTA per SM) owns one processed row at a time; CTA `rank`
+// owns a contiguous slice of the vocabulary, cut into chunks of at most 512 16-byte pieces per
+// array.  Two sweeps are made over the slice: sweep 1 accumulates the log-sum-exp statistics of
+// both rows and sum e*delta (plus, for rows without a gradient, the moments of its squared norm);
+// sweep 2 writes the gradient with 16-byte coalesced stores.
 //
-// Ring invariant: chunks are numbered q = 0,1,2,... in the order rows are processed; chunk q lives
-// in slot q % nslot and is fill number q / nslot of that slot.  full[slot] completes once per fill
-// (producer arrive + transaction bytes), empty[slot] once per drain (one arrive per consumer warp).
-// Per-row hand-offs are double buffered by row parity: partready (consumers -> finisher, sweep-1
-// partials), rowready (finisher -> consumers, row scalars), qready (consumers -> finisher, squared
-// norm of the written gradient), xbar (peer finishers -> finisher, exchanged records).
+// What bounds a streaming kernel is the number of bytes it keeps in flight (memory latency x
+// bandwidth is about 60 KB per SM), so shared memory is split between two uses:
+//   * `nres` chunks of the slice are RESIDENT: loaded once, read by sweep 1, kept, read again by
+//     sweep 2 and only then handed back;
+//   * the other chunks are STREAMED through a ring of `nring` slots that is always free to take
+//     new loads: sweep 1 consumes and releases them, sweep 2 fetches them a second time -- a few
+//     microseconds after the first read, so the second fetch is served by the L2 cache, not HBM.
+// Resident and streamed chunks alternate along the slice, so HBM reads are in flight during both
+// sweeps: the streamed part of row i during sweep 1 of row i, the resident part of row i+1 during
+// sweep 2 of row i.  Two producer warps issue the bulk asynchronous copies (cp.async.bulk, one
+// mbarrier per slot): one feeds the ring, one refills the resident slots.
 //
-// Every wait is bounded by a wall-clock limit; on expiry the CTA raises ADWIN_DEV_TIMEOUT, stops
-// waiting anywhere, drains its own copies, and still reaches the final cluster barrier so that no
-// peer is left behind.
+// 16 consumer warps do the arithmetic, each at its own pace: nothing but data dependences ties
+// them together.  Exponentials are taken against a reference that the whole row shares (the
+// logit of the sampled token), so partial sums add without rescaling.  After sweep 1 every warp
+// writes its partial record into the exchange buffer of every CTA of the cluster (remote shared
+// memory stores + remote mbarrier arrive), waits for the cl*16 records of the row, and sums them
+// in a fixed order: all warps of all CTAs obtain bit-identical totals and derive the row's
+// scalars themselves, with no hop through a leader.  Records also carry each warp's share of the
+// squared norm of the gradient row written before.  If the sums overflow the shared reference (a
+// sampled token more than ~27 nats below the row maximum), the cluster re-reads the row from
+// global memory with a running maximum and exchanges once more.
+//
+// Clusters are persistent and walk the compact list of in-window rows; rows past the window cost
+// nothing.  Every wait is bounded by a wall-clock limit; on expiry the CTA raises
+// ADWIN_DEV_TIMEOUT, stops waiting anywhere, drains its own copies, and still reaches the final
+// cluster barrier so that no peer is left behind.
 #include <mutex>
 #include <vector>
 
@@ -39,20 +43,26 @@ namespace adwin {
 
 constexpr int kNT = 512;             // consumer threads
 constexpr int kNW = kNT / 32;        // consumer warps
-constexpr int kProducerWarp = kNW;
-constexpr int kFinisherWarp = kNW + 1;
-constexpr int kThreads = kNT + 64;   // + producer warp + finisher warp
-constexpr int kMaxSlots = 32;
-constexpr int kMaxCL = 8;
-constexpr int kXF = 12;              // floats per exchange record
-constexpr int kCtrlBytes = 4096;
+constexpr int kG = 2;                // consumer groups: group g takes the chunks j with j % kG == g
+constexpr int kGT = kNT / kG;        // threads per group; each handles kG pieces of a chunk
+constexpr int kGW = kNW / kG;        // warps per group = arrivals that release a slot
+constexpr int kMaxChunks = 256;
+constexpr int kRingWarp = kNW;       // producer of the stream ring
+constexpr int kResWarp = kNW + 1;    // producer of the resident slots
+constexpr int kThreads = kNT + 64;
+constexpr int kMaxRes = 16;
+constexpr int kMaxRing = 16;
+constexpr int kMaxCL = 4;
+constexpr int kMaxRec = kMaxCL * kNW;  // exchange records per row
+constexpr int kCtrlBytes = 8192;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+constexpr float kSumLimit = 1.0995116e12f;        // 2^40: beyond it the shared reference is unsafe
 
 struct StagedPlan {
   int cl;                 // cluster size
-  int lag;                // 1: sweep 2 runs one row behind sweep 1 (two row slices resident)
-  int nslot;              // ring slots
   int nch;                // chunks per slice (same for every rank)
+  int nres;               // resident chunks per slice
+  int nring;              // stream-ring slots
   int chunk_pieces;       // 16-byte pieces per chunk (per array)
   int per_rank_pieces;    // pieces per slice (last rank may own fewer)
   int num_clusters;
@@ -60,18 +70,17 @@ struct StagedPlan {
 };
 
 struct __align__(16) Ctrl {
-  unsigned long long full[kMaxSlots];
-  unsigned long long empty[kMaxSlots];
+  unsigned long long res_full[kMaxRes];
+  unsigned long long res_empty[kMaxRes];
+  unsigned long long ring_full[kMaxRing];
+  unsigned long long ring_empty[kMaxRing];
   unsigned long long xbar[2];
-  unsigned long long partready[2];
-  unsigned long long qready[2];
-  unsigned long long rowready[2];
+  unsigned long long sbar;
   int abort_flag;
-  int pad[3];
-  float xbuf[2][kMaxCL][kXF];
-  float wpart[2][kNW][8];
-  float wq[2][kNW];
-  float rowres[2][8];
+  int pad;
+  float xbuf[2][kMaxRec][8];   // per row parity: one record per (rank, warp)
+  float sbuf[kMaxRec][8];      // records of the running-maximum fallback
+  int16_t tab[kMaxChunks];     // chunk j -> resident slot k (>= 0) or -1 (streamed)
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
@@ -175,15 +184,6 @@ __device__ __forceinline__ int64_t locate_row(const KlParams& p, int64_t n, int6
   return b * p.T + (n - p.offsets[b]);
 }
 
-template <typename TIn>
-__device__ __forceinline__ void load_piece(const char* slot, uint32_t u_off, int piece,
-                                           float (&z)[Elem<TIn>::N], float (&u)[Elem<TIn>::N]) {
-  const uint4 zv = *reinterpret_cast<const uint4*>(slot + (size_t)piece * 16);
-  const uint4 uv = *reinterpret_cast<const uint4*>(slot + u_off + (size_t)piece * 16);
-  Elem<TIn>::unpack(zv, z);
-  Elem<TIn>::unpack(uv, u);
-}
-
 // ---------------------------------------------------------------------------- packed fp32 pairs
 // sm_100 issues add/mul/fma on two fp32 lanes held in a 64-bit register pair in one slot
 // (add.f32x2 / mul.f32x2 / fma.f32x2).  The sweeps are issue- and MUFU-bound, so all element-wise
@@ -250,74 +250,35 @@ struct Pairs<float> {
 // Per-thread accumulators of one row slice, as pairs (even / odd entries).
 struct Acc2 {
   f2_t S, A, St, B0, B1, B2;
-  float m2s, m2t;
   __device__ __forceinline__ void reset() {
     S = A = St = B0 = B1 = B2 = 0ull;   // the bit pattern of {0.f, 0.f}
-    m2s = -INFINITY;
-    m2t = -INFINITY;
   }
 };
 
+// Sweep 1, rows whose gradient is written: e = 2^(z log2e - ref_s), delta = z - u uncentred.
 template <int NP>
-__device__ __forceinline__ void piece_max(const f2_t (&Z)[NP], const f2_t (&U)[NP], float& zm,
-                                          float& um) {
-  zm = -INFINITY;
-  um = -INFINITY;
-#pragma unroll
-  for (int i = 0; i < NP; ++i) {
-    float a, b;
-    upk2(Z[i], a, b);
-    zm = fmaxf(zm, fmaxf(a, b));
-    upk2(U[i], a, b);
-    um = fmaxf(um, fmaxf(a, b));
-  }
-}
-
-// Rows whose gradient is written: fixed references (set from the thread's first piece), no
-// per-piece maximum, delta = z - u uncentred.  The caller checks the sums for overflow after the
-// sweep and, if a later entry ran more than ~2^100 above the reference, redoes the slice with the
-// online-maximum path (the slice is still resident in shared memory).
-template <int NP>
-__device__ __forceinline__ void acc_fast(const f2_t (&Z)[NP], const f2_t (&U)[NP], f2_t nm2s,
-                                         f2_t nm2t, Acc2& a) {
+__device__ __forceinline__ void acc_grad(const f2_t (&Z)[NP], const f2_t (&U)[NP], f2_t nrefs,
+                                         f2_t nreft, Acc2& a) {
   const f2_t L2 = splat2(kLog2e), NEG1 = splat2(-1.f);
 #pragma unroll
   for (int i = 0; i < NP; ++i) {
-    const f2_t E = ex2_2(fma2(Z[i], L2, nm2s));
+    const f2_t E = ex2_2(fma2(Z[i], L2, nrefs));
     const f2_t D = fma2(U[i], NEG1, Z[i]);
     a.S = add2(a.S, E);
     a.A = fma2(E, D, a.A);
-    a.St = add2(a.St, ex2_2(fma2(U[i], L2, nm2t)));
+    a.St = add2(a.St, ex2_2(fma2(U[i], L2, nreft)));
   }
 }
 
-// Rows whose gradient is not written (probe rows): online maximum per piece, plus the moments
+// Sweep 1, rows whose gradient is not written (probe rows): additionally the moments
 // sum e^2 {1, delta, delta^2} of the single-sweep squared gradient norm, delta centred on dref.
 template <int NP>
-__device__ __forceinline__ void acc_probe(const f2_t (&Z)[NP], const f2_t (&U)[NP], float dref,
-                                          Acc2& a) {
-  float zm, um;
-  piece_max<NP>(Z, U, zm, um);
-  const float zl = zm * kLog2e, ul = um * kLog2e;
-  if (zl > a.m2s) {
-    const float f = ex2f(a.m2s - zl);
-    const f2_t F = splat2(f), F2 = splat2(f * f);
-    a.S = mul2(a.S, F);
-    a.A = mul2(a.A, F);
-    a.B0 = mul2(a.B0, F2);
-    a.B1 = mul2(a.B1, F2);
-    a.B2 = mul2(a.B2, F2);
-    a.m2s = zl;
-  }
-  if (ul > a.m2t) {
-    a.St = mul2(a.St, splat2(ex2f(a.m2t - ul)));
-    a.m2t = ul;
-  }
+__device__ __forceinline__ void acc_probe(const f2_t (&Z)[NP], const f2_t (&U)[NP], f2_t nrefs,
+                                          f2_t nreft, f2_t ndref, Acc2& a) {
   const f2_t L2 = splat2(kLog2e), NEG1 = splat2(-1.f);
-  const f2_t nm2s = splat2(-a.m2s), nm2t = splat2(-a.m2t), ndref = splat2(-dref);
 #pragma unroll
   for (int i = 0; i < NP; ++i) {
-    const f2_t E = ex2_2(fma2(Z[i], L2, nm2s));
+    const f2_t E = ex2_2(fma2(Z[i], L2, nrefs));
     const f2_t D = add2(fma2(U[i], NEG1, Z[i]), ndref);
     a.S = add2(a.S, E);
     a.A = fma2(E, D, a.A);
@@ -326,7 +287,7 @@ __device__ __forceinline__ void acc_probe(const f2_t (&Z)[NP], const f2_t (&U)[N
     a.B0 = add2(a.B0, E2);
     a.B1 = add2(a.B1, E2D);
     a.B2 = fma2(E2D, D, a.B2);
-    a.St = add2(a.St, ex2_2(fma2(U[i], L2, nm2t)));
+    a.St = add2(a.St, ex2_2(fma2(U[i], L2, nreft)));
   }
 }
 
@@ -355,8 +316,8 @@ __device__ __forceinline__ void store_pairs(char* dst, const f2_t (&G)[NP]) {
   }
 }
 
-// Row metadata shared by the consumer and finisher roles: which global row, whether its gradient
-// is written, its sampled token and the two logits at that token.
+// Row metadata: which global row, whether its gradient is written, its sampled token and the
+// two logits at that token (at element 0 when the token is out of range).
 struct RowCursor {
   int64_t b;   // monotone sequence pointer
   __device__ __forceinline__ void fetch_row(const KlParams& p, int64_t ordinal, bool in_range,
@@ -379,20 +340,35 @@ __device__ __forceinline__ void fetch_logits_at(const KlParams& p, int64_t r, in
   uy = Elem<TIn>::load1(static_cast<const char*>(p.teacher) + (size_t)r * p.ld * sizeof(TIn), yi);
 }
 
+// Chunk j of a slice is resident iff the running count floor(j*nres/nch) steps at j: the nres
+// resident chunks are spread evenly along the slice.  Returns the resident slot or -1.
+__device__ __forceinline__ int resident_slot(int j, int nres, int nch) {
+  const int a = (j * nres) / nch, b = ((j + 1) * nres) / nch;
+  return b > a ? a : -1;
+}
+
+// Fixed-order sum over the lanes of a warp; every lane returns the same bits.
+__device__ __forceinline__ float lane_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
 template <typename TIn, typename TOut>
 __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, StagedPlan plan) {
   constexpr int N = Elem<TIn>::N;
   constexpr int NP = Pairs<TIn>::NP;
   extern __shared__ __align__(128) char smem[];
   Ctrl& ctrl = *reinterpret_cast<Ctrl*>(smem);
-  char* ring = smem + kCtrlBytes;
+  char* res_base = smem + kCtrlBytes;
+  char* ring_base = res_base + (size_t)plan.nres * plan.slot_bytes;
   volatile int* abort = &ctrl.abort_flag;
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_rank();
   const int cl = plan.cl;
-  const int lag = plan.lag;
+  const int nch = plan.nch, nres = plan.nres, nring = plan.nring;
   const int64_t cluster_id = blockIdx.x / cl;
   const uint32_t u_off = (uint32_t)plan.chunk_pieces * 16u;
 
@@ -407,16 +383,18 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       cluster_id < total_rows ? (total_rows - cluster_id + plan.num_clusters - 1) / plan.num_clusters : 0;
 
   if (tid == 0) {
-    for (int s = 0; s < plan.nslot; ++s) {
-      mbar_init(smem_u32(&ctrl.full[s]), 1);
-      mbar_init(smem_u32(&ctrl.empty[s]), kNW);
+    for (int s = 0; s < nres; ++s) {
+      mbar_init(smem_u32(&ctrl.res_full[s]), 1);
+      mbar_init(smem_u32(&ctrl.res_empty[s]), kGW);
     }
-    for (int k = 0; k < 2; ++k) {
-      mbar_init(smem_u32(&ctrl.xbar[k]), cl);
-      mbar_init(smem_u32(&ctrl.partready[k]), kNW);
-      mbar_init(smem_u32(&ctrl.qready[k]), kNW);
-      mbar_init(smem_u32(&ctrl.rowready[k]), 1);
+    for (int s = 0; s < nring; ++s) {
+      mbar_init(smem_u32(&ctrl.ring_full[s]), 1);
+      mbar_init(smem_u32(&ctrl.ring_empty[s]), kGW);
     }
+    for (int j = 0; j < nch; ++j) ctrl.tab[j] = (int16_t)resident_slot(j, nres, nch);
+    mbar_init(smem_u32(&ctrl.xbar[0]), cl * kNW);
+    mbar_init(smem_u32(&ctrl.xbar[1]), cl * kNW);
+    mbar_init(smem_u32(&ctrl.sbar), cl * kNW);
     ctrl.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -428,52 +406,60 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
     const int left = (int)my_pieces - j * plan.chunk_pieces;
     return left < plan.chunk_pieces ? left : plan.chunk_pieces;
   };
+  // issue the two bulk copies of chunk j of row r into a slot
+  auto issue_chunk = [&](int64_t r, int j, char* slot, unsigned long long* full) {
+    int np = pieces_in_chunk(j);
+    np = np < 0 ? 0 : np;
+    const uint32_t bytes = (uint32_t)np * 16u;
+    const uint32_t bar = smem_u32(full);
+    if (bytes == 0) {
+      mbar_arrive(bar);
+    } else {
+      const size_t goff = ((size_t)r * p.ld + (size_t)piece0 * N) * sizeof(TIn) +
+                          (size_t)j * plan.chunk_pieces * 16;
+      mbar_arrive_expect_tx(bar, 2u * bytes);
+      const uint32_t dst = smem_u32(slot);
+      bulk_load(dst, static_cast<const char*>(p.student) + goff, bytes, bar);
+      bulk_load(dst + u_off, static_cast<const char*>(p.teacher) + goff, bytes, bar);
+    }
+  };
 
-  if (warp == kProducerWarp) {
-    // ------------------------------------------------------------------ producer warp
-    if (lane == 0) {
+  if (warp == kRingWarp) {
+    // ------------------------------------------------------------------ ring producer
+    // Order of the stream: per row, the streamed chunks for sweep 1, then (rows whose gradient is
+    // written) the same chunks again for sweep 2.
+    if (lane == 0 && nring > 0 && nres < nch) {
       int slot = 0;
       uint32_t phase = 0;
       int64_t fills = 0;
       int64_t b = 0;
-      for (int64_t i = 0; i < my_rows; ++i) {
-        if (*abort) break;
+      for (int64_t i = 0; i < my_rows && !*abort; ++i) {
         const int64_t r = locate_row(p, cluster_id + i * plan.num_clusters, b);
-        const char* zrow = static_cast<const char*>(p.student) + ((size_t)r * p.ld + piece0 * N) * sizeof(TIn);
-        const char* urow = static_cast<const char*>(p.teacher) + ((size_t)r * p.ld + piece0 * N) * sizeof(TIn);
-        for (int j = 0; j < plan.nch; ++j) {
-          if (fills >= plan.nslot) bounded_wait<false>(smem_u32(&ctrl.empty[slot]), phase ^ 1u, abort);
-          int np = pieces_in_chunk(j);
-          np = np < 0 ? 0 : np;
-          const uint32_t bytes = (uint32_t)np * 16u;
-          const uint32_t bar = smem_u32(&ctrl.full[slot]);
-          if (bytes == 0) {
-            mbar_arrive(bar);
-          } else {
-            mbar_arrive_expect_tx(bar, 2u * bytes);
-            const uint32_t dst = smem_u32(ring + (size_t)slot * plan.slot_bytes);
-            const size_t goff = (size_t)j * plan.chunk_pieces * 16;
-            bulk_load(dst, zrow + goff, bytes, bar);
-            bulk_load(dst + u_off, urow + goff, bytes, bar);
-          }
-          ++fills;
-          if (++slot == plan.nslot) {
-            slot = 0;
-            phase ^= 1u;
+        const int64_t bb = r / p.T;
+        const bool wg = (p.grad != nullptr) && ((r - bb * p.T) < p.ewin[bb]);
+        for (int sweep = 0; sweep < (wg ? 2 : 1); ++sweep) {
+          for (int j = 0; j < nch; ++j) {
+            if (ctrl.tab[j] >= 0) continue;
+            if (fills >= nring) bounded_wait<false>(smem_u32(&ctrl.ring_empty[slot]), phase ^ 1u, abort);
+            issue_chunk(r, j, ring_base + (size_t)slot * plan.slot_bytes, &ctrl.ring_full[slot]);
+            ++fills;
+            if (++slot == nring) {
+              slot = 0;
+              phase ^= 1u;
+            }
           }
         }
       }
       // Drain: every copy this CTA issued must have landed before its shared memory goes away.
-      // Walk back over the last min(fills, nslot) fills.
-      int64_t pending = fills < plan.nslot ? fills : plan.nslot;
+      int64_t pending = fills < nring ? fills : nring;
       const uint64_t t0 = global_timer();
       bool gave_up = false;
       while (pending > 0) {
         if (--slot < 0) {
-          slot = plan.nslot - 1;
+          slot = nring - 1;
           phase ^= 1u;
         }
-        const uint32_t bar = smem_u32(&ctrl.full[slot]);
+        const uint32_t bar = smem_u32(&ctrl.ring_full[slot]);
         while (!gave_up && !mbar_try_wait(bar, phase)) {
           if (global_timer() - t0 > kWaitLimitNs) gave_up = true;
         }
@@ -481,22 +467,63 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       }
       if (gave_up) atomicOr(p.status, ADWIN_DEV_TIMEOUT);
     }
-  } else if (warp == kFinisherWarp) {
-    // ------------------------------------------------------------------ finisher warp
-    // Iteration i < my_rows exchanges the sweep-1 record of row i; every iteration also carries the
-    // CTA's share of the squared gradient norm of row i-1-lag (written by sweep 2), so 1+lag
-    // trailing iterations deliver the last norms.  All CTAs of a cluster run the same iterations.
+  } else if (warp == kResWarp) {
+    // ------------------------------------------------------------------ resident producer
+    // Resident slot k takes resident chunk k of every row: fill number i belongs to row i and
+    // waits for drain number i-1 (sweep 2 of row i-1, or its sweep 1 if no gradient is written).
+    if (lane == 0 && nres > 0) {
+      int64_t b = 0;
+      int64_t done = 0;
+      for (int64_t i = 0; i < my_rows && !*abort; ++i) {
+        const int64_t r = locate_row(p, cluster_id + i * plan.num_clusters, b);
+        for (int j = 0; j < nch; ++j) {
+          const int k = ctrl.tab[j];
+          if (k < 0) continue;
+          if (i > 0)
+            bounded_wait<false>(smem_u32(&ctrl.res_empty[k]), (uint32_t)((i - 1) & 1), abort);
+          issue_chunk(r, j, res_base + (size_t)k * plan.slot_bytes, &ctrl.res_full[k]);
+        }
+        done = i + 1;
+      }
+      if (done > 0) {   // drain the last fill of every resident slot
+        const uint64_t t0 = global_timer();
+        bool gave_up = false;
+        for (int k = 0; k < nres; ++k) {
+          const uint32_t bar = smem_u32(&ctrl.res_full[k]);
+          while (!gave_up && !mbar_try_wait(bar, (uint32_t)((done - 1) & 1))) {
+            if (global_timer() - t0 > kWaitLimitNs) gave_up = true;
+          }
+        }
+        if (gave_up) atomicOr(p.status, ADWIN_DEV_TIMEOUT);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ consumer warps
+    const bool full_mode = (p.mode == ADWIN_GRAD_FULL_KL);
+    const int nrec = cl * kNW;
+    int rc_slot = 0;            // ring cursor
+    uint32_t rc_phase = 0;
+    uint32_t safe_rounds = 0;   // completed fallback exchanges (parity of sbar)
+    bool timed_out = false;
+    float q_prev = 0.f;         // this warp's share of the previous written row's squared norm
+    int64_t r_prev = 0;
+    bool wg_prev = false;
+
+    // metadata pipeline: current row (C) and next row (N) held in registers
     RowCursor cur;
     cur.b = 0;
-    int64_t rC = 0, rN = 0, rH1 = 0, rH2 = 0;
+    int64_t rC = 0, rN = 0;
     int yC = 0, yN = 0;
     float zyC = 0.f, uyC = 0.f;
-    bool wgC = false, wgN = false, wgH1 = false, wgH2 = false;
+    bool wgC = false, wgN = false;
     cur.fetch_row(p, cluster_id, 0 < my_rows, rC, yC, wgC);
     if (my_rows > 0) fetch_logits_at<TIn>(p, rC, yC, zyC, uyC);
     cur.fetch_row(p, cluster_id + plan.num_clusters, 1 < my_rows, rN, yN, wgN);
-    bool timed_out = false;
-    const int64_t iters = my_rows > 0 ? my_rows + 1 + lag : 0;
+
+    const int grp = warp / kGW;                  // this warp's group: chunks j % kG == grp
+    const int gt = tid - grp * kGT;              // thread index inside the group
+    const uint32_t toff = (uint32_t)gt * 16u;    // first of this thread's kG pieces in a chunk
+    const int64_t iters = my_rows > 0 ? my_rows + 1 : 0;   // + one exchange for the last norm
     for (int64_t i = 0; i < iters; ++i) {
       const bool real = i < my_rows;
       // next rows' dependent loads, consumed one iteration later
@@ -507,298 +534,243 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       if (i + 1 < my_rows) fetch_logits_at<TIn>(p, rN, yN, zyN, uyN);
       cur.fetch_row(p, cluster_id + (i + 2) * plan.num_clusters, i + 2 < my_rows, rNN, yNN, wgNN);
 
-      const int par = (int)(i & 1);
-      const uint32_t ph = (uint32_t)((i >> 1) & 1);
-      float rec[8] = {-INFINITY, 0.f, 0.f, 0.f, 0.f, 0.f, -INFINITY, 0.f};
+      const bool y_valid = (yC >= 0) && ((int64_t)yC < p.V);
+      const float ref_s = zyC * kLog2e, ref_t = uyC * kLog2e;   // shared references of the row
+      const float dref = wgC ? 0.f : zyC - uyC;                 // delta is centred on probe rows
+      const uint32_t rpar = (uint32_t)(i & 1);                  // fill parity of resident slots
+
+      // ---------------------------------------------------------------- sweep 1
+      Acc2 a;
+      a.reset();
       if (real) {
-        if (!bounded_wait<false>(smem_u32(&ctrl.partready[par]), ph, abort)) {
-          timed_out = true;
-          break;
-        }
-        // combine the consumer warps of this CTA (lane = source warp)
-        const bool has = lane < kNW;
-        const float* w = ctrl.wpart[par][has ? lane : 0];
-        const float ms = has ? w[0] : -INFINITY, mt = has ? w[6] : -INFINITY;
-        const float Ms = warp_max(ms), Mt = warp_max(mt);
-        const float fs = (ms == -INFINITY) ? 0.f : ex2f(ms - Ms);
-        const float ft = (mt == -INFINITY) ? 0.f : ex2f(mt - Mt);
-        const float fs2 = fs * fs;
-        rec[0] = Ms;
-        rec[1] = warp_sum(has ? w[1] * fs : 0.f);
-        rec[2] = warp_sum(has ? w[2] * fs : 0.f);
-        rec[3] = warp_sum(has ? w[3] * fs2 : 0.f);
-        rec[4] = warp_sum(has ? w[4] * fs2 : 0.f);
-        rec[5] = warp_sum(has ? w[5] * fs2 : 0.f);
-        rec[6] = Mt;
-        rec[7] = warp_sum(has ? w[7] * ft : 0.f);
-      }
-      const int64_t jq = i - 1 - lag;               // row whose written-gradient norm is carried
-      const int64_t rq = lag ? rH2 : rH1;
-      const bool wgq = lag ? wgH2 : wgH1;
-      float qcta = 0.f;
-      if (jq >= 0) {
-        if (!bounded_wait<false>(smem_u32(&ctrl.qready[jq & 1]), (uint32_t)((jq >> 1) & 1), abort)) {
-          timed_out = true;
-          break;
-        }
-        qcta = warp_sum(lane < kNW ? ctrl.wq[jq & 1][lane] : 0.f);
-      }
-      // exchange: lane d delivers this CTA's record to peer d, then arrives on d's barrier
-      if (lane < cl) {
-        const uint32_t dst = map_to_rank(smem_u32(&ctrl.xbuf[par][rank][0]), (uint32_t)lane);
-        remote_store4(dst, rec[0], rec[1], rec[2], rec[3]);
-        remote_store4(dst + 16, rec[4], rec[5], rec[6], rec[7]);
-        remote_store4(dst + 32, qcta, 0.f, 0.f, 0.f);
-        remote_arrive_release(map_to_rank(smem_u32(&ctrl.xbar[par]), (uint32_t)lane));
-      }
-      if (!bounded_wait<true>(smem_u32(&ctrl.xbar[par]), ph, abort)) {
-        timed_out = true;
-        break;
-      }
-      // combine the CL records (lane = source rank); identical in every CTA of the cluster
-      RowTotals t;
-      float qtot;
-      {
-        const bool has = lane < cl;
-        const float* x = ctrl.xbuf[par][has ? lane : 0];
-        const float ms = has ? x[0] : -INFINITY, mt = has ? x[6] : -INFINITY;
-        t.M2s = warp_max(ms);
-        t.M2t = warp_max(mt);
-        const float fs = (ms == -INFINITY) ? 0.f : ex2f(ms - t.M2s);
-        const float ft = (mt == -INFINITY) ? 0.f : ex2f(mt - t.M2t);
-        const float fs2 = fs * fs;
-        t.S = warp_sum(has ? x[1] * fs : 0.f);
-        t.A = warp_sum(has ? x[2] * fs : 0.f);
-        t.B0 = warp_sum(has ? x[3] * fs2 : 0.f);
-        t.B1 = warp_sum(has ? x[4] * fs2 : 0.f);
-        t.B2 = warp_sum(has ? x[5] * fs2 : 0.f);
-        t.St = warp_sum(has ? x[7] * ft : 0.f);
-        qtot = warp_sum(has ? x[8] : 0.f);
-      }
-      if (lane == 0) {
-        if (rank == 0 && jq >= 0 && wgq && p.gsq) p.gsq[rq] = qtot;
-        if (real) {
-          const bool y_valid = (yC >= 0) && ((int64_t)yC < p.V);
-          const float dref = wgC ? 0.f : zyC - uyC;   // sweep 1 centres delta only on probe rows
-          const RowScalars rs = finish_row(t, zyC, uyC, y_valid, dref, p.alpha, p.mode);
-          float* rr = ctrl.rowres[par];
-          rr[0] = t.M2s;
-          rr[1] = rs.c0;
-          rr[2] = rs.coef;
-          rr[3] = rs.gy;
-          if (rank == 0) {
-            p.kl[rC] = rs.kl;
-            p.logratio[rC] = rs.c;
-            if (p.gsq && !wgC) p.gsq[rC] = rs.gsq_expanded;
-            if (p.lse_s) p.lse_s[rC] = rs.lse_s;
-            if (p.lse_t) p.lse_t[rC] = rs.lse_t;
-            int bits = 0;
-            if (!y_valid) bits |= ADWIN_DEV_TOKEN_RANGE;
-            if (rs.nonfinite) bits |= ADWIN_DEV_NONFINITE;
-            if (bits) atomicOr(p.status, bits);
-          }
-          mbar_arrive(smem_u32(&ctrl.rowready[par]));   // release: the row scalars are visible
-        }
-      }
-      __syncwarp();
-      // rotate the metadata pipeline
-      rH2 = rH1; wgH2 = wgH1;
-      rH1 = rC; wgH1 = wgC;
-      rC = rN; yC = yN; wgC = wgN; zyC = zyN; uyC = uyN;
-      rN = rNN; yN = yNN; wgN = wgNN;
-    }
-    if (timed_out && lane == 0) {
-      atomicOr(p.status, ADWIN_DEV_TIMEOUT);
-      for (int d = 0; d < cl; ++d)
-        remote_store_u32(map_to_rank(smem_u32(&ctrl.abort_flag), (uint32_t)d), 1u);
-    }
-  } else {
-    // ------------------------------------------------------------------ consumer warps
-    const bool full_mode = (p.mode == ADWIN_GRAD_FULL_KL);
-    int s1_slot = 0, s2_slot = 0;
-    uint32_t s1_phase = 0;
-    bool timed_out = false;
-
-    // metadata pipeline: row of this iteration's sweep 1 (C), the next one (N), the previous (P)
-    RowCursor cur;
-    cur.b = 0;
-    int64_t rC = 0, rN = 0, rP = 0;
-    int yC = 0, yN = 0, yP = 0;
-    float zyC = 0.f, uyC = 0.f;
-    bool wgC = false, wgN = false, wgP = false;
-    cur.fetch_row(p, cluster_id, 0 < my_rows, rC, yC, wgC);
-    if (my_rows > 0) fetch_logits_at<TIn>(p, rC, yC, zyC, uyC);
-    cur.fetch_row(p, cluster_id + plan.num_clusters, 1 < my_rows, rN, yN, wgN);
-
-    const uint32_t toff = (uint32_t)tid * 16u;   // this thread's piece inside every chunk
-    const int64_t iters = my_rows > 0 ? my_rows + lag : 0;
-    for (int64_t i = 0; i < iters; ++i) {
-      float zyN = 0.f, uyN = 0.f;
-      int64_t rNN = 0;
-      int yNN = 0;
-      bool wgNN = false;
-      if (i + 1 < my_rows) fetch_logits_at<TIn>(p, rN, yN, zyN, uyN);
-      cur.fetch_row(p, cluster_id + (i + 2) * plan.num_clusters, i + 2 < my_rows, rNN, yNN, wgNN);
-
-      // ---------------------------------------------------------------- sweep 1 of row i
-      if (i < my_rows) {
-        Acc2 a;
-        a.reset();
-        const int slot0 = s1_slot;
-        if (wgC) {
-          // gradient row: fixed references from the first piece, checked once after the sweep
-          f2_t nm2s = 0ull, nm2t = 0ull;
-          bool have_ref = false;
-          for (int j = 0; j < plan.nch; ++j) {
-            if (!bounded_wait<false>(smem_u32(&ctrl.full[s1_slot]), s1_phase, abort)) timed_out = true;
-            if (tid < pieces_in_chunk(j)) {
-              const char* sl = ring + (size_t)s1_slot * plan.slot_bytes + toff;
-              f2_t Z[NP], U[NP];
-              Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl), Z);
-              Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl + u_off), U);
-              if (!have_ref) {
-                float zm, um;
-                piece_max<NP>(Z, U, zm, um);
-                a.m2s = zm * kLog2e;
-                a.m2t = um * kLog2e;
-                nm2s = splat2(-a.m2s);
-                nm2t = splat2(-a.m2t);
-                have_ref = true;
+        const f2_t nrefs = splat2(-ref_s), nreft = splat2(-ref_t), ndref = splat2(-dref);
+        for (int j = 0; j < nch; ++j) {
+          const int k = ctrl.tab[j];
+          if (j % kG == grp) {
+            const char* sl;
+            if (k >= 0) {
+              if (!bounded_wait<false>(smem_u32(&ctrl.res_full[k]), rpar, abort)) timed_out = true;
+              sl = res_base + (size_t)k * plan.slot_bytes + toff;
+            } else {
+              if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort)) timed_out = true;
+              sl = ring_base + (size_t)rc_slot * plan.slot_bytes + toff;
+            }
+            if (timed_out) break;
+            const int np = pieces_in_chunk(j);
+#pragma unroll
+            for (int h = 0; h < kG; ++h) {
+              if (gt + h * kGT < np) {
+                f2_t Z[NP], U[NP];
+                Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl + h * kGT * 16), Z);
+                Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl + u_off + h * kGT * 16), U);
+                if (wgC)
+                  acc_grad<NP>(Z, U, nrefs, nreft, a);
+                else
+                  acc_probe<NP>(Z, U, nrefs, nreft, ndref, a);
               }
-              acc_fast<NP>(Z, U, nm2s, nm2t, a);
             }
-            if (++s1_slot == plan.nslot) {
-              s1_slot = 0;
-              s1_phase ^= 1u;
+            if (k < 0 || !wgC) {
+              __syncwarp();
+              if (lane == 0)
+                mbar_arrive(smem_u32(k < 0 ? &ctrl.ring_empty[rc_slot] : &ctrl.res_empty[k]));
             }
           }
-          // overflow / invalid reference: redo this thread's pieces with the online maximum
-          constexpr float kSumLimit = 1.2676506e30f;   // 2^100
-          if (!(hsum2(a.S) < kSumLimit) || !(hsum2(a.St) < kSumLimit)) {
-            RowAcc ra;
-            ra.reset();
-            int s = slot0;
-            for (int j = 0; j < plan.nch; ++j) {
-              if (tid < pieces_in_chunk(j)) {
-                float z[N], u[N];
-                load_piece<TIn>(ring + (size_t)s * plan.slot_bytes, u_off, tid, z, u);
-                acc_piece<N, false>(z, u, 0.f, ra);
-              }
-              if (++s == plan.nslot) s = 0;
-            }
-            a.reset();
-            a.m2s = ra.m2s;
-            a.m2t = ra.m2t;
-            a.S = pk2(ra.S, 0.f);
-            a.A = pk2(ra.A, 0.f);
-            a.St = pk2(ra.St, 0.f);
-          }
-        } else {
-          // probe row: nothing re-reads a chunk, so each slot goes back to the producer at once
-          const float dref = zyC - uyC;
-          for (int j = 0; j < plan.nch; ++j) {
-            if (!bounded_wait<false>(smem_u32(&ctrl.full[s1_slot]), s1_phase, abort)) timed_out = true;
-            if (tid < pieces_in_chunk(j)) {
-              const char* sl = ring + (size_t)s1_slot * plan.slot_bytes + toff;
-              f2_t Z[NP], U[NP];
-              Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl), Z);
-              Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl + u_off), U);
-              acc_probe<NP>(Z, U, dref, a);
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctrl.empty[s1_slot]));
-            if (++s1_slot == plan.nslot) {
-              s1_slot = 0;
-              s1_phase ^= 1u;
-            }
+          if (k < 0 && ++rc_slot == nring) {   // the ring cursor walks every streamed chunk
+            rc_slot = 0;
+            rc_phase ^= 1u;
           }
         }
         if (timed_out) break;
-        // warp partials -> finisher
-        const float wms = warp_max(a.m2s), wmt = warp_max(a.m2t);
-        const float fs = (a.m2s == -INFINITY) ? 0.f : ex2f(a.m2s - wms);
-        const float ft = (a.m2t == -INFINITY) ? 0.f : ex2f(a.m2t - wmt);
-        const float fs2 = fs * fs;
-        const float v0 = warp_sum(hsum2(a.S) * fs), v1 = warp_sum(hsum2(a.A) * fs);
-        const float v2 = warp_sum(hsum2(a.B0) * fs2), v3 = warp_sum(hsum2(a.B1) * fs2);
-        const float v4 = warp_sum(hsum2(a.B2) * fs2), v5 = warp_sum(hsum2(a.St) * ft);
-        if (lane == 0) {
-          float* w = ctrl.wpart[i & 1][warp];
-          w[0] = wms; w[1] = v0; w[2] = v1; w[3] = v2; w[4] = v3; w[5] = v4; w[6] = wmt; w[7] = v5;
-          mbar_arrive(smem_u32(&ctrl.partready[i & 1]));
-        }
       }
 
-      // ---------------------------------------------------------------- sweep 2 of row i - lag
-      const int64_t j2 = i - lag;
-      if (j2 >= 0) {
-        const int64_t r2 = lag ? rP : rC;
-        const int y2 = lag ? yP : yC;
-        const bool wg2 = lag ? wgP : wgC;
-        const int par = (int)(j2 & 1);
-        if (!bounded_wait<false>(smem_u32(&ctrl.rowready[par]), (uint32_t)((j2 >> 1) & 1), abort)) {
+      // ---------------------------------------------------------------- exchange
+      // record = { S, A, St, B0, B1, B2, q_prev, 0 }: this warp's sums over its lanes.
+      RowTotals t;
+      float qtot;
+      {
+        const float v0 = lane_sum(hsum2(a.S)), v1 = lane_sum(hsum2(a.A)), v2 = lane_sum(hsum2(a.St));
+        float v3 = 0.f, v4 = 0.f, v5 = 0.f;
+        if (real && !wgC) {
+          v3 = lane_sum(hsum2(a.B0));
+          v4 = lane_sum(hsum2(a.B1));
+          v5 = lane_sum(hsum2(a.B2));
+        }
+        const int par = (int)(i & 1);
+        if (lane < cl) {
+          const uint32_t dst =
+              map_to_rank(smem_u32(&ctrl.xbuf[par][rank * kNW + warp][0]), (uint32_t)lane);
+          remote_store4(dst, v0, v1, v2, v3);
+          remote_store4(dst + 16, v4, v5, q_prev, 0.f);
+          remote_arrive_release(map_to_rank(smem_u32(&ctrl.xbar[par]), (uint32_t)lane));
+        }
+        if (!bounded_wait<true>(smem_u32(&ctrl.xbar[par]), (uint32_t)((i >> 1) & 1), abort)) {
           timed_out = true;
           break;
         }
-        float q = 0.f;
-        if (wg2) {
-          const float M2s = ctrl.rowres[par][0], c0 = ctrl.rowres[par][1], coef = ctrl.rowres[par][2],
-                      gy = ctrl.rowres[par][3];
-          const bool y_valid = (y2 >= 0) && ((int64_t)y2 < p.V);
-          const f2_t L2 = splat2(kLog2e), NEG1 = splat2(-1.f);
-          const f2_t nM2s = splat2(-M2s), nc0 = splat2(-c0), coef2 = splat2(coef);
-          const int64_t ypiece = y_valid ? ((int64_t)y2 / N - piece0) : -1;   // slice-relative
-          char* gthread = static_cast<char*>(p.grad) +
-                          ((size_t)r2 * p.ld_grad + (size_t)(piece0 + tid) * N) * sizeof(TOut);
-          const size_t gstep = (size_t)plan.chunk_pieces * N * sizeof(TOut);
-          f2_t Q = 0ull;
-          for (int j = 0; j < plan.nch; ++j) {
-            if (tid < pieces_in_chunk(j)) {
-              const char* sl = ring + (size_t)s2_slot * plan.slot_bytes + toff;
-              f2_t Z[NP], U[NP], G[NP];
-              Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl), Z);
-              Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl + u_off), U);
-#pragma unroll
-              for (int k = 0; k < NP; ++k) {
-                const f2_t E = ex2_2(fma2(Z[k], L2, nM2s));
-                if (full_mode) {
-                  const f2_t D = add2(fma2(U[k], NEG1, Z[k]), nc0);
-                  G[k] = mul2(E, mul2(D, coef2));
-                } else {
-                  G[k] = mul2(E, coef2);
-                }
-              }
-              if (!full_mode && (int64_t)j * plan.chunk_pieces + tid == ypiece) {
-                const int e = (int)((int64_t)y2 - ((int64_t)y2 / N) * N);
-#pragma unroll
-                for (int k = 0; k < NP; ++k) {
-                  float lo, hi;
-                  upk2(G[k], lo, hi);
-                  if (e == 2 * k) lo = gy;
-                  if (e == 2 * k + 1) hi = gy;
-                  G[k] = pk2(lo, hi);
-                }
-              }
-#pragma unroll
-              for (int k = 0; k < NP; ++k) Q = fma2(G[k], G[k], Q);
-              store_pairs<TOut, NP>(gthread + (size_t)j * gstep, G);
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctrl.empty[s2_slot]));
-            if (++s2_slot == plan.nslot) s2_slot = 0;
-          }
-          q = warp_sum(hsum2(Q));
-        } else {
-          s2_slot = (s2_slot + plan.nch) % plan.nslot;   // released by sweep 1 already
+        // fixed-order sum of the nrec records (lane = record, then a butterfly)
+        float s[7] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int rr = lane; rr < nrec; rr += 32) {
+          const float4 x0 = *reinterpret_cast<const float4*>(&ctrl.xbuf[par][rr][0]);
+          const float4 x1 = *reinterpret_cast<const float4*>(&ctrl.xbuf[par][rr][4]);
+          s[0] += x0.x; s[1] += x0.y; s[2] += x0.z; s[3] += x0.w;
+          s[4] += x1.x; s[5] += x1.y; s[6] += x1.z;
         }
-        if (lane == 0) {
-          ctrl.wq[par][warp] = q;
-          mbar_arrive(smem_u32(&ctrl.qready[par]));
+        t.M2s = ref_s;
+        t.M2t = ref_t;
+        t.S = lane_sum(s[0]);
+        t.A = lane_sum(s[1]);
+        t.St = lane_sum(s[2]);
+        t.B0 = t.B1 = t.B2 = 0.f;
+        if (real && !wgC) {
+          t.B0 = lane_sum(s[3]);
+          t.B1 = lane_sum(s[4]);
+          t.B2 = lane_sum(s[5]);
         }
+        qtot = lane_sum(s[6]);
+      }
+      if (warp == 0 && lane == 0 && rank == 0 && i > 0 && wg_prev && p.gsq) p.gsq[r_prev] = qtot;
+      if (!real) break;
+
+      // ---------------------------------------------------------------- overflow fallback
+      // The totals are identical in every warp of the cluster, so this branch is uniform.
+      if (!(t.S < kSumLimit) || !(t.St < kSumLimit) || !(t.B0 < kSumLimit)) {
+        RowAcc ra;
+        ra.reset();
+        const char* zrow = static_cast<const char*>(p.student) + ((size_t)rC * p.ld + (size_t)piece0 * N) * sizeof(TIn);
+        const char* urow = static_cast<const char*>(p.teacher) + ((size_t)rC * p.ld + (size_t)piece0 * N) * sizeof(TIn);
+        for (int64_t pc = tid; pc < my_pieces; pc += kNT) {
+          float z[N], u[N];
+          const uint4 zv = __ldg(reinterpret_cast<const uint4*>(zrow) + pc);
+          const uint4 uv = __ldg(reinterpret_cast<const uint4*>(urow) + pc);
+          Elem<TIn>::unpack(zv, z);
+          Elem<TIn>::unpack(uv, u);
+          acc_piece<N, true>(z, u, dref, ra);
+        }
+        const float wms = warp_max(ra.m2s), wmt = warp_max(ra.m2t);
+        const float fs = (ra.m2s == -INFINITY) ? 0.f : ex2f(ra.m2s - wms);
+        const float ft = (ra.m2t == -INFINITY) ? 0.f : ex2f(ra.m2t - wmt);
+        const float fs2 = fs * fs;
+        const float w1 = lane_sum(ra.S * fs), w2 = lane_sum(ra.A * fs), w3 = lane_sum(ra.B0 * fs2);
+        const float w4 = lane_sum(ra.B1 * fs2), w5 = lane_sum(ra.B2 * fs2), w7 = lane_sum(ra.St * ft);
+        if (lane < cl) {
+          const uint32_t dst = map_to_rank(smem_u32(&ctrl.sbuf[rank * kNW + warp][0]), (uint32_t)lane);
+          remote_store4(dst, wms, w1, w2, w3);
+          remote_store4(dst + 16, w4, w5, wmt, w7);
+          remote_arrive_release(map_to_rank(smem_u32(&ctrl.sbar), (uint32_t)lane));
+        }
+        if (!bounded_wait<true>(smem_u32(&ctrl.sbar), safe_rounds & 1u, abort)) {
+          timed_out = true;
+          break;
+        }
+        ++safe_rounds;
+        float ms = -INFINITY, mt = -INFINITY;
+        for (int rr = lane; rr < nrec; rr += 32) {
+          ms = fmaxf(ms, ctrl.sbuf[rr][0]);
+          mt = fmaxf(mt, ctrl.sbuf[rr][6]);
+        }
+        t.M2s = warp_max(ms);
+        t.M2t = warp_max(mt);
+        float s[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int rr = lane; rr < nrec; rr += 32) {
+          const float* x = ctrl.sbuf[rr];
+          const float gs = (x[0] == -INFINITY) ? 0.f : ex2f(x[0] - t.M2s);
+          const float gt = (x[6] == -INFINITY) ? 0.f : ex2f(x[6] - t.M2t);
+          const float gs2 = gs * gs;
+          s[0] += x[1] * gs; s[1] += x[2] * gs; s[2] += x[3] * gs2;
+          s[3] += x[4] * gs2; s[4] += x[5] * gs2; s[5] += x[7] * gt;
+        }
+        t.S = lane_sum(s[0]);
+        t.A = lane_sum(s[1]);
+        t.B0 = lane_sum(s[2]);
+        t.B1 = lane_sum(s[3]);
+        t.B2 = lane_sum(s[4]);
+        t.St = lane_sum(s[5]);
       }
 
+      // ---------------------------------------------------------------- row scalars
+      const RowScalars rs = finish_row(t, zyC, uyC, y_valid, dref, p.alpha, p.mode);
+      if (warp == 0 && lane == 0 && rank == 0) {
+        p.kl[rC] = rs.kl;
+        p.logratio[rC] = rs.c;
+        if (p.gsq && !wgC) p.gsq[rC] = rs.gsq_expanded;
+        if (p.lse_s) p.lse_s[rC] = rs.lse_s;
+        if (p.lse_t) p.lse_t[rC] = rs.lse_t;
+        int bits = 0;
+        if (!y_valid) bits |= ADWIN_DEV_TOKEN_RANGE;
+        if (rs.nonfinite) bits |= ADWIN_DEV_NONFINITE;
+        if (bits) atomicOr(p.status, bits);
+      }
+
+      // ---------------------------------------------------------------- sweep 2
+      q_prev = 0.f;
+      if (wgC) {
+        const f2_t L2 = splat2(kLog2e), NEG1 = splat2(-1.f);
+        const f2_t nM2s = splat2(-t.M2s), nc0 = splat2(-rs.c0), coef2 = splat2(rs.coef);
+        const int64_t ypiece = y_valid ? ((int64_t)yC / N - piece0) : -1;   // slice-relative
+        char* gthread = static_cast<char*>(p.grad) +
+                        ((size_t)rC * p.ld_grad + (size_t)(piece0 + gt) * N) * sizeof(TOut);
+        const size_t gstep = (size_t)plan.chunk_pieces * N * sizeof(TOut);
+        f2_t Q = 0ull;
+        for (int j = 0; j < nch; ++j) {
+          const int k = ctrl.tab[j];
+          if (j % kG == grp) {
+            const char* sl;
+            if (k >= 0) {
+              sl = res_base + (size_t)k * plan.slot_bytes + toff;   // still there since sweep 1
+            } else {
+              if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort)) timed_out = true;
+              sl = ring_base + (size_t)rc_slot * plan.slot_bytes + toff;
+            }
+            if (timed_out) break;
+            const int np = pieces_in_chunk(j);
+#pragma unroll
+            for (int h = 0; h < kG; ++h) {
+              if (gt + h * kGT < np) {
+                f2_t Z[NP], U[NP], G[NP];
+                Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl + h * kGT * 16), Z);
+                Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl + u_off + h * kGT * 16), U);
+#pragma unroll
+                for (int e = 0; e < NP; ++e) {
+                  const f2_t E = ex2_2(fma2(Z[e], L2, nM2s));
+                  if (full_mode) {
+                    const f2_t D = add2(fma2(U[e], NEG1, Z[e]), nc0);
+                    G[e] = mul2(E, mul2(D, coef2));
+                  } else {
+                    G[e] = mul2(E, coef2);
+                  }
+                }
+                if (!full_mode && (int64_t)j * plan.chunk_pieces + gt + h * kGT == ypiece) {
+                  const int e = (int)((int64_t)yC - ((int64_t)yC / N) * N);
+#pragma unroll
+                  for (int w = 0; w < NP; ++w) {
+                    float lo, hi;
+                    upk2(G[w], lo, hi);
+                    if (e == 2 * w) lo = rs.gy;
+                    if (e == 2 * w + 1) hi = rs.gy;
+                    G[w] = pk2(lo, hi);
+                  }
+                }
+#pragma unroll
+                for (int e = 0; e < NP; ++e) Q = fma2(G[e], G[e], Q);
+                store_pairs<TOut, NP>(gthread + (size_t)j * gstep + (size_t)h * kGT * N * sizeof(TOut), G);
+              }
+            }
+            __syncwarp();
+            if (lane == 0)
+              mbar_arrive(smem_u32(k < 0 ? &ctrl.ring_empty[rc_slot] : &ctrl.res_empty[k]));
+          }
+          if (k < 0 && ++rc_slot == nring) {
+            rc_slot = 0;
+            rc_phase ^= 1u;
+          }
+        }
+        if (timed_out) break;
+        q_prev = lane_sum(hsum2(Q));
+      }
+      r_prev = rC;
+      wg_prev = wgC;
+
       // rotate the metadata pipeline
-      rP = rC; yP = yC; wgP = wgC;
       rC = rN; yC = yN; wgC = wgN; zyC = zyN; uyC = uyN;
       rN = rNN; yN = yNN; wgN = wgNN;
     }
@@ -818,48 +790,56 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
 namespace {
 
 constexpr int kSmemOptin = 232448;   // 227 KB: the per-CTA limit of sm_100
+// Streamed chunks are read a second time by sweep 2; the bytes of one round of rows that have to
+// survive in L2 until then should stay well inside the cache.
+constexpr double kL2BudgetBytes = 32.0 * 1024 * 1024;
 
-// Chunking of one cluster size; false when the slice does not fit the ring.
+// Chunking and the resident / streamed split for one cluster size.
 bool plan_for_cluster(int64_t pieces_total, int cl, bool has_grad, StagedPlan& plan) {
-  const int64_t ring_bytes = kSmemOptin - kCtrlBytes;
+  const int64_t slots_bytes = kSmemOptin - kCtrlBytes;
   const int64_t per_rank = (pieces_total + cl - 1) / cl;
   if (per_rank * 16 > (int64_t)1 << 30) return false;
-  int64_t nch, chunk_pieces;
-  if (has_grad) {
-    nch = (per_rank + kNT - 1) / kNT;
-    chunk_pieces = (per_rank + nch - 1) / nch;
-  } else {
-    chunk_pieces = per_rank < kNT ? per_rank : kNT;
-    nch = (per_rank + chunk_pieces - 1) / chunk_pieces;
-  }
+  int64_t nch = (per_rank + kNT - 1) / kNT;
+  int64_t chunk_pieces = (per_rank + nch - 1) / nch;
   chunk_pieces = (chunk_pieces + 7) / 8 * 8;   // slots start on 128-byte boundaries
   if (chunk_pieces > kNT) chunk_pieces = kNT;
   nch = (per_rank + chunk_pieces - 1) / chunk_pieces;
+  if (nch > kMaxChunks) return false;
   const int64_t slot_bytes = 2 * chunk_pieces * 16;
-  int64_t nslot = ring_bytes / slot_bytes;
-  if (nslot > kMaxSlots) nslot = kMaxSlots;
-  int lag = 0;
-  if (has_grad) {
-    if (2 * nch + 1 <= nslot) lag = 1;          // two row slices resident + one slot in flight
-    else if (nch + 2 > nslot) return false;     // one row slice + two slots in flight
+  const int64_t nslot = slots_bytes / slot_bytes;
+  if (nslot < 2) return false;
+  int64_t nres = 0, nring = 0;
+  if (!has_grad) {
+    nring = nslot < kMaxRing ? nslot : kMaxRing;   // nothing is read twice
   } else {
-    if (nslot < 2) return false;
-    lag = 1;   // no slot is held for a second sweep: only the wait for the row scalars is deferred
+    // About 0.42 of the slice resident balances the HBM reads of the two sweeps (sweep 1 takes
+    // ~1.6x as long as sweep 2); the rest of the slots form the ring.
+    nres = (nch * 42 + 50) / 100;
+    if (nres > kMaxRes) nres = kMaxRes;
+    if (nres > nslot - 2) nres = nslot - 2;
+    if (nres < 0) nres = 0;
+    nring = nslot - nres;
+    if (nring > kMaxRing) nring = kMaxRing;
+    if (nres == nch) nring = 0;                    // everything resident: no stream
   }
   plan.cl = cl;
-  plan.lag = lag;
-  plan.nslot = (int)nslot;
   plan.nch = (int)nch;
+  plan.nres = (int)nres;
+  plan.nring = (int)nring;
   plan.chunk_pieces = (int)chunk_pieces;
   plan.per_rank_pieces = (int)per_rank;
   plan.slot_bytes = (uint32_t)slot_bytes;
   return true;
 }
 
+int plan_smem_bytes(const StagedPlan& plan) {
+  return kCtrlBytes + (plan.nres + plan.nring) * (int)plan.slot_bytes;
+}
+
 template <typename TIn, typename TOut>
 cudaError_t max_clusters_for(const StagedPlan& plan, int sm_count, int& max_clusters) {
   auto kernel = kl_staged_kernel<TIn, TOut>;
-  const int smem = kCtrlBytes + plan.nslot * (int)plan.slot_bytes;
+  const int smem = plan_smem_bytes(plan);
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
@@ -876,9 +856,9 @@ cudaError_t max_clusters_for(const StagedPlan& plan, int sm_count, int& max_clus
   return cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg);
 }
 
-// The cluster size is chosen once per (device, shape class): among the sizes whose slice fits,
-// prefer plans that hide the exchange (lag 1), then the one that keeps the most SMs busy (cluster
-// sizes that do not divide a GPC's SM count leave SMs idle), then the smaller cluster.
+// The cluster size is chosen once per (device, shape class): the one that keeps the most SMs busy
+// (cluster sizes that do not divide a GPC's SM count leave SMs idle) among those whose streamed
+// bytes fit the L2 budget, else the one with the fewest streamed bytes.
 struct PlanKey {
   int dev, dtype, grad_dtype, has_grad;
   int64_t pieces_total;
@@ -906,7 +886,10 @@ bool choose_plan(int64_t pieces_total, bool has_grad, int sm_count, StagedPlan& 
     }
     if (clusters < 1) continue;
     const double ctas = (double)clusters * cl;
-    const double score = ctas * ((plan.lag || !has_grad) ? 1.0 : 0.6) - 1e-3 * cl;
+    const double streamed = ctas * (double)(plan.nch - plan.nres) * plan.slot_bytes;
+    double score = ctas;
+    if (has_grad && streamed > kL2BudgetBytes) score *= kL2BudgetBytes / streamed;
+    score -= 1e-3 * cl;
     if (score > best_score) {
       best_score = score;
       best = plan;
@@ -946,7 +929,7 @@ cudaError_t launch_staged_t(const KlParams& p, int dtype, int grad_dtype, int sm
   if (!ok) return cudaErrorNotSupported;
 
   auto kernel = kl_staged_kernel<TIn, TOut>;
-  const int smem = kCtrlBytes + plan.nslot * (int)plan.slot_bytes;
+  const int smem = plan_smem_bytes(plan);
   e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};

@@ -112,6 +112,23 @@ def test_dtype_combinations_and_grad_scale(path, in_dt, g_dt):
                       flags=PATHS[path] | api.ZERO_TAIL)
 
 
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("in_dt,g_dt", [(2, torch.bfloat16), (1, torch.float32), (2, None)])
+def test_sampled_token_far_below_the_row_maximum(path, in_dt, g_dt):
+    """Rows whose sampled token has a vanishing probability (the staged kernel's shared reference
+    overflows there and the row is redone with a running maximum), next to ordinary rows."""
+    batch = synth.make_batch(in_dt, device=DEV, B=2, T=6, V=8192)
+    batch.window = torch.tensor([6, 4], dtype=torch.int32, device=DEV)
+    for (b, t, gap_s, gap_t) in [(0, 1, 90.0, 0.0), (0, 3, 0.0, 120.0), (1, 2, 60.0, 70.0),
+                                 (1, 5, 200.0, 200.0)]:
+        y = int(batch.tokens[b, t])
+        batch.student[b, t, y] = batch.student[b, t].float().max() - gap_s
+        batch.teacher[b, t, y] = batch.teacher[b, t].float().max() - gap_t
+    flags = PATHS[path] | (api.RANGE_FULL if g_dt is None else 0)
+    run_and_check(batch, grad_dtype=g_dt, flags=flags)
+    run_and_check(batch, grad_dtype=g_dt, grad_mode=api.GRAD_SAMPLED, flags=flags)
+
+
 @pytest.mark.parametrize("V", [1, 2, 7, 8, 9, 1001, 4100, 65537])
 def test_odd_vocab_sizes(V):
     batch = synth.make_batch(2, device=DEV, B=2, T=6, V=V)
