@@ -43,9 +43,9 @@ namespace adwin {
 
 constexpr int kNT = 512;             // consumer threads
 constexpr int kNW = kNT / 32;        // consumer warps
-constexpr int kG = 2;                // consumer groups: group g takes the chunks j with j % kG == g
+constexpr int kG = 4;                // consumer groups: group g takes the chunks j with j % kG == g
 constexpr int kGT = kNT / kG;        // threads per group; each handles kG pieces of a chunk
-constexpr int kGW = kNW / kG;        // warps per group = arrivals that release a slot
+constexpr int kGW = kNW / kG;        // warps per group = arrivals that release a resident slot
 constexpr int kMaxChunks = 256;
 constexpr int kRingWarp = kNW;       // producer of the stream ring
 constexpr int kResWarp = kNW + 1;    // producer of the resident slots
@@ -389,7 +389,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
     }
     for (int s = 0; s < nring; ++s) {
       mbar_init(smem_u32(&ctrl.ring_full[s]), 1);
-      mbar_init(smem_u32(&ctrl.ring_empty[s]), kGW);
+      mbar_init(smem_u32(&ctrl.ring_empty[s]), kNW);
     }
     for (int j = 0; j < nch; ++j) ctrl.tab[j] = (int16_t)resident_slot(j, nres, nch);
     mbar_init(smem_u32(&ctrl.xbar[0]), cl * kNW);
@@ -433,14 +433,19 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       uint32_t phase = 0;
       int64_t fills = 0;
       int64_t b = 0;
-      for (int64_t i = 0; i < my_rows && !*abort; ++i) {
+      bool stop = false;
+      for (int64_t i = 0; i < my_rows && !stop && !*abort; ++i) {
         const int64_t r = locate_row(p, cluster_id + i * plan.num_clusters, b);
         const int64_t bb = r / p.T;
         const bool wg = (p.grad != nullptr) && ((r - bb * p.T) < p.ewin[bb]);
-        for (int sweep = 0; sweep < (wg ? 2 : 1); ++sweep) {
+        for (int sweep = 0; sweep < (wg ? 2 : 1) && !stop; ++sweep) {
           for (int j = 0; j < nch; ++j) {
             if (ctrl.tab[j] >= 0) continue;
-            if (fills >= nring) bounded_wait<false>(smem_u32(&ctrl.ring_empty[slot]), phase ^ 1u, abort);
+            if (fills >= nring &&
+                !bounded_wait<false>(smem_u32(&ctrl.ring_empty[slot]), phase ^ 1u, abort)) {
+              stop = true;   // gave up: never overwrite a slot that may still be read
+              break;
+            }
             issue_chunk(r, j, ring_base + (size_t)slot * plan.slot_bytes, &ctrl.ring_full[slot]);
             ++fills;
             if (++slot == nring) {
@@ -473,29 +478,34 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
     // waits for drain number i-1 (sweep 2 of row i-1, or its sweep 1 if no gradient is written).
     if (lane == 0 && nres > 0) {
       int64_t b = 0;
-      int64_t done = 0;
+      int64_t last_row = -1;   // last row some slot was filled for, and how many slots got it
+      int last_k = 0;
       for (int64_t i = 0; i < my_rows && !*abort; ++i) {
         const int64_t r = locate_row(p, cluster_id + i * plan.num_clusters, b);
         for (int j = 0; j < nch; ++j) {
           const int k = ctrl.tab[j];
           if (k < 0) continue;
-          if (i > 0)
-            bounded_wait<false>(smem_u32(&ctrl.res_empty[k]), (uint32_t)((i - 1) & 1), abort);
+          if (i > 0 &&
+              !bounded_wait<false>(smem_u32(&ctrl.res_empty[k]), (uint32_t)((i - 1) & 1), abort))
+            break;   // gave up: never overwrite a slot that may still be read
           issue_chunk(r, j, res_base + (size_t)k * plan.slot_bytes, &ctrl.res_full[k]);
+          last_row = i;
+          last_k = k + 1;
         }
-        done = i + 1;
       }
-      if (done > 0) {   // drain the last fill of every resident slot
-        const uint64_t t0 = global_timer();
-        bool gave_up = false;
-        for (int k = 0; k < nres; ++k) {
-          const uint32_t bar = smem_u32(&ctrl.res_full[k]);
-          while (!gave_up && !mbar_try_wait(bar, (uint32_t)((done - 1) & 1))) {
-            if (global_timer() - t0 > kWaitLimitNs) gave_up = true;
-          }
+      // Drain: the last fill of every resident slot must have landed before the CTA exits
+      // (slots k < last_k were filled for last_row, the others for the row before).
+      const uint64_t t0 = global_timer();
+      bool gave_up = false;
+      for (int k = 0; k < nres; ++k) {
+        const int64_t fill = k < last_k ? last_row : last_row - 1;
+        if (fill < 0) continue;
+        const uint32_t bar = smem_u32(&ctrl.res_full[k]);
+        while (!gave_up && !mbar_try_wait(bar, (uint32_t)(fill & 1))) {
+          if (global_timer() - t0 > kWaitLimitNs) gave_up = true;
         }
-        if (gave_up) atomicOr(p.status, ADWIN_DEV_TIMEOUT);
       }
+      if (gave_up) atomicOr(p.status, ADWIN_DEV_TIMEOUT);
     }
   } else {
     // ------------------------------------------------------------------ consumer warps
@@ -574,6 +584,14 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
               if (lane == 0)
                 mbar_arrive(smem_u32(k < 0 ? &ctrl.ring_empty[rc_slot] : &ctrl.res_empty[k]));
             }
+          } else if (k < 0) {
+            // Not this group's chunk, but every warp observes and releases every fill of a ring
+            // slot: a parity wait is only sound within one phase of the barrier's current one.
+            if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort)) {
+              timed_out = true;
+              break;
+            }
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl.ring_empty[rc_slot]));
           }
           if (k < 0 && ++rc_slot == nring) {   // the ring cursor walks every streamed chunk
             rc_slot = 0;
@@ -758,6 +776,12 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
             __syncwarp();
             if (lane == 0)
               mbar_arrive(smem_u32(k < 0 ? &ctrl.ring_empty[rc_slot] : &ctrl.res_empty[k]));
+          } else if (k < 0) {
+            if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort)) {
+              timed_out = true;
+              break;
+            }
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl.ring_empty[rc_slot]));
           }
           if (k < 0 && ++rc_slot == nring) {
             rc_slot = 0;
