@@ -1,7 +1,7 @@
 // Staged cluster kernel: each logit byte is read from HBM once.
 //
 // A thread-block cluster of CL CTAs (one CTA per SM) owns one processed row at a time; CTA `rank`
-// owns a contiguous slice of the vocabulary, cut into chunks of at most 512 16-byte pieces per
+// owns a contiguous slice of the vocabulary, cut into chunks of at most 1536 16-byte pieces per
 // array.  Two sweeps are made over the slice: sweep 1 accumulates the log-sum-exp statistics of
 // both rows and sum e*delta (plus, for rows without a gradient, the moments of its squared norm);
 // sweep 2 writes the gradient with 16-byte coalesced stores.
@@ -43,9 +43,11 @@ namespace adwin {
 
 constexpr int kNT = 512;             // consumer threads
 constexpr int kNW = kNT / 32;        // consumer warps
-constexpr int kG = 4;                // consumer groups: group g takes the chunks j with j % kG == g
-constexpr int kGT = kNT / kG;        // threads per group; each handles kG pieces of a chunk
+constexpr int kG = 1;                // consumer groups: group g takes the chunks j with j % kG == g
+constexpr int kP = 3;                // pieces of a chunk that each thread of the owning group handles
+constexpr int kGT = kNT / kG;        // threads per group
 constexpr int kGW = kNW / kG;        // warps per group = arrivals that release a resident slot
+constexpr int kChunkMax = kGT * kP;  // 16-byte pieces per chunk (per array), at most
 constexpr int kMaxChunks = 256;
 constexpr int kRingWarp = kNW;       // producer of the stream ring
 constexpr int kResWarp = kNW + 1;    // producer of the resident slots
@@ -532,7 +534,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
 
     const int grp = warp / kGW;                  // this warp's group: chunks j % kG == grp
     const int gt = tid - grp * kGT;              // thread index inside the group
-    const uint32_t toff = (uint32_t)gt * 16u;    // first of this thread's kG pieces in a chunk
+    const uint32_t toff = (uint32_t)gt * 16u;    // first of this thread's kP pieces in a chunk
     const int64_t iters = my_rows > 0 ? my_rows + 1 : 0;   // + one exchange for the last norm
     for (int64_t i = 0; i < iters; ++i) {
       const bool real = i < my_rows;
@@ -568,7 +570,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
             if (timed_out) break;
             const int np = pieces_in_chunk(j);
 #pragma unroll
-            for (int h = 0; h < kG; ++h) {
+            for (int h = 0; h < kP; ++h) {
               if (gt + h * kGT < np) {
                 f2_t Z[NP], U[NP];
                 Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl + h * kGT * 16), Z);
@@ -742,7 +744,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
             if (timed_out) break;
             const int np = pieces_in_chunk(j);
 #pragma unroll
-            for (int h = 0; h < kG; ++h) {
+            for (int h = 0; h < kP; ++h) {
               if (gt + h * kGT < np) {
                 f2_t Z[NP], U[NP], G[NP];
                 Pairs<TIn>::make(*reinterpret_cast<const uint4*>(sl + h * kGT * 16), Z);
@@ -823,10 +825,10 @@ bool plan_for_cluster(int64_t pieces_total, int cl, bool has_grad, StagedPlan& p
   const int64_t slots_bytes = kSmemOptin - kCtrlBytes;
   const int64_t per_rank = (pieces_total + cl - 1) / cl;
   if (per_rank * 16 > (int64_t)1 << 30) return false;
-  int64_t nch = (per_rank + kNT - 1) / kNT;
+  int64_t nch = (per_rank + kChunkMax - 1) / kChunkMax;
   int64_t chunk_pieces = (per_rank + nch - 1) / nch;
   chunk_pieces = (chunk_pieces + 7) / 8 * 8;   // slots start on 128-byte boundaries
-  if (chunk_pieces > kNT) chunk_pieces = kNT;
+  if (chunk_pieces > kChunkMax) chunk_pieces = kChunkMax;
   nch = (per_rank + chunk_pieces - 1) / chunk_pieces;
   if (nch > kMaxChunks) return false;
   const int64_t slot_bytes = 2 * chunk_pieces * 16;
@@ -840,7 +842,7 @@ bool plan_for_cluster(int64_t pieces_total, int cl, bool has_grad, StagedPlan& p
     // ~1.6x as long as sweep 2); the rest of the slots form the ring.
     nres = (nch * 42 + 50) / 100;
     if (nres > kMaxRes) nres = kMaxRes;
-    if (nres > nslot - 2) nres = nslot - 2;
+    if (nres > nslot - 3) nres = nslot - 3;      // the ring keeps at least three slots in flight
     if (nres < 0) nres = 0;
     nring = nslot - nres;
     if (nring > kMaxRing) nring = kMaxRing;
