@@ -232,7 +232,7 @@ void adwin_oracle_window_reduce(const double *kl, const double *logratio, const 
  *   batch_stats[j]   = { rho_micro, rho_macro, snr_micro, admissible (0/1), n_tokens }
  * macro = mean over all B sequences of rho_b (per-sample cosines averaged); micro = the cosine
  * after summing over the batch (Figure 5).  SNR = rho^2 / (1 - rho^2); admissible when
- * rho_micro >= rho_star (Eq. 5, inclusive).  L_next = the smallest candidate length that is
+ * rho_micro >= rho_star (threshold equation of Section 4.2, inclusive).  L_next = the smallest candidate length that is
  * admissible (Section 4.2); when none is, the largest candidate and flag NONE_ADMISSIBLE.
  * A zero full norm gives rho = 1 (prefix and full gradients coincide) and flag DEGENERATE.
  */
