@@ -144,7 +144,7 @@ int adwin_window_reduce(const float* kl, const float* logratio, const float* gsq
  *   seq_full    [B,3]     = { Q_b_full, sum kl, sum logratio over t < R_b }
  *   batch_stats [K+1,5]   = { rho_micro, rho_macro, snr_micro, admissible (0/1), n_tokens }
  * rho_macro = mean over the B sequences of rho_b; rho_micro = the cosine after batch aggregation
- * (Figure 5); SNR = rho^2/(1-rho^2); admissible <=> rho_micro >= rho_star (Eq. 5, inclusive).
+ * (Figure 5); SNR = rho^2/(1-rho^2); admissible <=> rho_micro >= rho_star (threshold equation of Section 4.2, inclusive).
  * *L_next = the smallest admissible candidate (the scheduler rule of Section 4.2), or the largest
  * candidate with ADWIN_ALIGN_NONE_ADMISSIBLE.  A zero full norm gives rho = 1 and
  * ADWIN_ALIGN_DEGENERATE.
@@ -185,6 +185,39 @@ int adwin_opd_kl_fwd_bwd_host(const void* student_host, const void* teacher_host
                               float* kl_host, float* logratio_host, float* gsq_host,
                               void* staging_dev, size_t staging_bytes, int64_t rows_per_stage,
                               int32_t* dev_status, void* cuda_stream);
+
+/*
+ * adwin_opd_kl_fwd_bwd without a workspace argument and without any allocation.
+ *
+ * The paper has no counterpart for this entry point.  It is for callers that cannot supply
+ * scratch memory and must not allocate: a trainer whose framework has claimed the whole GPU for
+ * its own memory pool (a cudaMalloc there would fail, or take memory away from the pool), code
+ * that runs where an allocation's implicit device-wide synchronisation is not acceptable, and
+ * bindings from runtimes that expose no device allocator at all.  The row map that
+ * adwin_opd_kl_fwd_bwd keeps in `workspace` is kept here in a fixed array inside the library
+ * image (about 66 KB on every GPU that loads the library, held until the process exits).  The
+ * call itself allocates and frees nothing, on the device or through any library.
+ *
+ * Arguments, outputs, rounding and error behaviour are those of adwin_opd_kl_fwd_bwd, with
+ * `workspace` / `workspace_bytes` left out.  Differences:
+ *   - B may be at most adwin_no_alloc_max_sequences() (4096); a larger batch returns
+ *     ADWIN_ERR_WORKSPACE and enqueues nothing.  T and V are not limited by the array.
+ *   - The first call on each device looks up the array's device address (that device must be
+ *     current, as for every call).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Each call rewrites it completely before reading
+ *     it, so nothing carries over from one call to the next, but two calls whose kernels can
+ *     overlap on the GPU (different streams, no dependency between them) race on it and give
+ *     undefined results: keep calls to this entry point ordered on one stream, or use
+ *     adwin_opd_kl_fwd_bwd with separate workspaces.
+ */
+int64_t adwin_no_alloc_max_sequences(void);
+int adwin_opd_kl_fwd_bwd_no_alloc(const void* student_logits, const void* teacher_logits,
+                                  int dtype, int64_t B, int64_t T, int64_t V, int64_t ld,
+                                  const int32_t* tokens, const int32_t* window,
+                                  const int32_t* rollout_len, float grad_scale, int grad_mode,
+                                  int flags, void* grad_student, int grad_dtype, int64_t ld_grad,
+                                  float* kl, float* logratio, float* gsq, float* lse_student,
+                                  float* lse_teacher, int32_t* dev_status, void* cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -22,11 +22,12 @@ ZERO_TAIL, RANGE_FULL, FORCE_GENERIC = 1, 2, 4
 DEV_TOKEN_RANGE, DEV_NONFINITE, DEV_TIMEOUT, DEV_BOUNDS, DEV_WINDOW = 1, 2, 4, 8, 16
 ALIGN_DEGENERATE, ALIGN_NONE_ADMISSIBLE = 1, 2
 DEFAULT_CANDIDATES = (64, 128, 256, 512, 1024, 2048)   # Section 5.1, Training Details
-RHO_STAR = math.sqrt(2.0) / 2.0                          # Eq. 5
+RHO_STAR = math.sqrt(2.0) / 2.0                          # Section 4.2, threshold equation
 
 EXPORTS = ("adwin_version", "adwin_status_string", "adwin_workspace_bytes",
            "adwin_opd_kl_fwd_bwd", "adwin_window_reduce", "adwin_probe_align",
-           "adwin_host_staging_bytes", "adwin_opd_kl_fwd_bwd_host")
+           "adwin_host_staging_bytes", "adwin_opd_kl_fwd_bwd_host",
+           "adwin_no_alloc_max_sequences", "adwin_opd_kl_fwd_bwd_no_alloc")
 
 _lib = None
 
@@ -68,6 +69,11 @@ def lib():
         L.adwin_opd_kl_fwd_bwd_host.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, i64, vp, vp,
                                                 vp, f32, ctypes.c_int, ctypes.c_int, vp,
                                                 ctypes.c_int, i64, vp, vp, vp, vp, sz, i64, vp, vp]
+        L.adwin_no_alloc_max_sequences.restype = i64
+        L.adwin_opd_kl_fwd_bwd_no_alloc.restype = ctypes.c_int
+        L.adwin_opd_kl_fwd_bwd_no_alloc.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, i64, vp,
+                                                    vp, vp, f32, ctypes.c_int, ctypes.c_int, vp,
+                                                    ctypes.c_int, i64, vp, vp, vp, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -231,3 +237,29 @@ def adwin_opd_kl_fwd_bwd_host(student, teacher, tokens, window, rollout_len=None
             int(rows_per_stage), _ptr(dev_status), _stream(dev))
     _check(rc)
     return o
+
+
+def adwin_no_alloc_max_sequences() -> int:
+    return int(lib().adwin_no_alloc_max_sequences())
+
+
+def adwin_opd_kl_fwd_bwd_no_alloc(student, teacher, tokens, window, rollout_len, *, grad, kl,
+                                  logratio, gsq, dev_status, grad_scale=1.0,
+                                  grad_mode=GRAD_FULL_KL, flags=0, lse_s=None, lse_t=None):
+    """The same pass through the entry point that needs no workspace and allocates nothing.
+
+    For callers that own every buffer up front and may not allocate: all inputs AND outputs are
+    passed in (this wrapper creates no tensor either), the row map lives in a fixed array inside
+    the library.  B is limited to ``adwin_no_alloc_max_sequences()``; calls must stay ordered on
+    one stream (they share that array).  ``grad`` may be None.  Returns None; raises AdwinError.
+    """
+    B, T, V = student.shape
+    ld = student.stride(1) if T > 1 else (student.stride(0) if B > 1 else V)
+    ld_grad = 0
+    if grad is not None:
+        ld_grad = grad.stride(1) if T > 1 else (grad.stride(0) if B > 1 else V)
+    _check(lib().adwin_opd_kl_fwd_bwd_no_alloc(
+        _ptr(student), _ptr(teacher), _dtype_code(student.dtype), B, T, V, ld, _ptr(tokens),
+        _ptr(window), _ptr(rollout_len), float(grad_scale), int(grad_mode), int(flags), _ptr(grad),
+        _dtype_code(grad.dtype) if grad is not None else 0, ld_grad, _ptr(kl), _ptr(logratio),
+        _ptr(gsq), _ptr(lse_s), _ptr(lse_t), _ptr(dev_status), _stream(student.device)))
