@@ -1,35 +1,40 @@
-// Staged cluster kernel: each logit byte is read from HBM once and the two sweeps of the method
-// run concurrently on different warps.
+// Staged cluster kernel: each logit byte is read from HBM once.
 //
 // A thread-block cluster of CL CTAs (one CTA per SM) owns one processed row at a time; CTA `rank`
-// owns a contiguous slice of the vocabulary, cut into chunks.  A producer lane streams the
-// chunks of consecutive rows into a FIFO ring of shared-memory slots with bulk asynchronous copies
-// (cp.async.bulk, one mbarrier per slot).  The ring holds a whole row slice plus a few slots in
-// flight, so a chunk stays on chip from its first use to its last:
-//   * the SWEEP-1 warps (10 of the 15 consumer warps) read each chunk as it lands and accumulate
-//     the log-sum-exp statistics of both rows and sum e*delta (for rows without a gradient also
-//     the moments of its squared norm); after the last chunk of a row every warp writes its
-//     partial record into the exchange buffer of every CTA of the cluster (remote shared-memory
-//     stores + remote mbarrier arrive) and goes straight on to the next row;
-//   * the SWEEP-2 warps (the other 5) wait for the cl*10 records of a row, sum them in a fixed
-//     order -- all of them, in every CTA, obtain bit-identical totals -- derive the row's scalars
-//     and write the gradient from the chunks that are still in the ring, with 16-byte coalesced
-//     stores, one row behind sweep 1.
-// Sweep 1 needs two exponentials per entry and sweep 2 one, so the 10:5 split keeps the special-
-// function pipe evenly loaded, HBM reads (sweep 1 of row i+1) and writes (sweep 2 of row i) flow
-// at the same time, and the latency of the cluster exchange is hidden behind the other sweep.  A
-// slot returns to the producer once every consumer warp has copied its pieces into registers.
+// owns a contiguous slice of the vocabulary, cut into chunks of at most 1536 16-byte pieces per
+// array.  Two sweeps are made over the slice: sweep 1 accumulates the log-sum-exp statistics of
+// both rows and sum e*delta (plus, for rows without a gradient, the moments of its squared norm);
+// sweep 2 writes the gradient with 16-byte coalesced stores.
 //
-// Exponentials are taken against a reference that the whole row shares (the logit of the sampled
-// token), so partial sums add without rescaling.  If the sums overflow that reference, the
-// sweep-2 warps of the cluster re-read the row from global memory with a running maximum and
-// exchange once more among themselves.
+// What bounds a streaming kernel is the number of bytes it keeps in flight (memory latency x
+// bandwidth is about 60 KB per SM), so shared memory is split between two uses:
+//   * `nres` chunks of the slice are RESIDENT: loaded once, read by sweep 1, kept, read again by
+//     sweep 2 and only then handed back;
+//   * the other chunks are STREAMED through a ring of `nring` slots that is always free to take
+//     new loads: sweep 1 consumes and releases them, sweep 2 fetches them a second time -- a few
+//     microseconds after the first read, so the second fetch is served by the L2 cache, not HBM.
+// Resident and streamed chunks alternate along the slice, so HBM reads are in flight during both
+// sweeps: the streamed part of row i during sweep 1 of row i, the resident part of row i+1 during
+// sweep 2 of row i.  Two lanes of a producer warp issue the bulk asynchronous copies
+// (cp.async.bulk, one mbarrier per slot): one feeds the ring, one refills the resident slots.
+// A consumer warp copies its pieces of a chunk into registers and hands the slot back at once,
+// so the refill is in flight while the arithmetic runs.
+//
+// 15 consumer warps do the arithmetic, each at its own pace: nothing but data dependences ties
+// them together.  Exponentials are taken against a reference that the whole row shares (the
+// logit of the sampled token), so partial sums add without rescaling.  After sweep 1 every warp
+// writes its partial record into the exchange buffer of every CTA of the cluster (remote shared
+// memory stores + remote mbarrier arrive), waits for the cl*15 records of the row, and sums them
+// in a fixed order: all warps of all CTAs obtain bit-identical totals and derive the row's
+// scalars themselves, with no hop through a leader.  Records also carry each warp's share of the
+// squared norm of the gradient row written before.  If the sums overflow the shared reference (a
+// sampled token more than ~69 nats below the row maximum), the cluster re-reads the row from
+// global memory with a running maximum and exchanges once more.
 //
 // Clusters are persistent and walk the compact list of in-window rows; rows past the window cost
-// nothing.  An mbarrier parity wait is only sound within one phase of the barrier, so every
-// consumer warp observes every fill of every slot.  Every wait is bounded by a wall-clock limit;
-// on expiry the CTA raises ADWIN_DEV_TIMEOUT, stops waiting anywhere, drains its own copies, and
-// still reaches the final cluster barrier so that no peer is left behind.
+// nothing.  Every wait is bounded by a wall-clock limit; on expiry the CTA raises
+// ADWIN_DEV_TIMEOUT, stops waiting anywhere, drains its own copies, and still reaches the final
+// cluster barrier so that no peer is left behind.
 #include <mutex>
 #include <vector>
 
@@ -38,24 +43,29 @@
 
 namespace adwin {
 
-constexpr int kThreads = 512;        // 16 warps: the block keeps 128 registers per thread
-constexpr int kNC = 15;              // consumer warps; warp 15 hosts the producer lane
-constexpr int kProducerWarp = kNC;
-constexpr int kP1 = 3;               // pieces of a chunk per sweep-1 thread
-constexpr int kP2 = 6;               // pieces of a chunk per sweep-2 thread (two rounds of kP2/2)
-constexpr int kMaxSlots = 32;
-constexpr int kMaxCL = 8;
-constexpr int kMaxRec1 = kMaxCL * 10;   // sweep-1 exchange records per row (cl * ns1)
-constexpr int kMaxRec2 = kMaxCL * 5;    // sweep-2 records: squared norms, fallback (cl * ns2)
-constexpr int kCtrlBytes = 9216;
+constexpr int kNT = 480;             // consumer threads (512 in all: the block keeps 128 registers per thread)
+constexpr int kNW = kNT / 32;        // consumer warps
+constexpr int kG = 1;                // consumer groups: group g takes the chunks j with j % kG == g
+constexpr int kP = 3;                // pieces of a chunk that each thread of the owning group handles
+constexpr int kGT = kNT / kG;        // threads per group
+constexpr int kGW = kNW / kG;        // warps per group = arrivals that release a resident slot
+constexpr int kChunkMax = kGT * kP;  // 16-byte pieces per chunk (per array), at most
+constexpr int kMaxChunks = 256;
+constexpr int kProducerWarp = kNW;   // lane 0 feeds the stream ring, lane 1 refills the resident slots
+constexpr int kThreads = kNT + 32;
+constexpr int kMaxRes = 16;
+constexpr int kMaxRing = 16;
+constexpr int kMaxCL = 4;
+constexpr int kMaxRec = kMaxCL * kNW;  // exchange records per row
+constexpr int kCtrlBytes = 8192;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
 constexpr float kSumLimit = 1.2676506e30f;        // 2^100: beyond it the shared reference is unsafe
 
 struct StagedPlan {
   int cl;                 // cluster size
-  int ns1, ns2;           // sweep-1 warps [0,ns1) and sweep-2 warps [ns1, ns1+ns2), ns1+ns2 == kNC
   int nch;                // chunks per slice (same for every rank)
-  int nslot;              // ring slots, <= 2 * nch - 1; >= nch + 1 when a gradient is written
+  int nres;               // resident chunks per slice
+  int nring;              // stream-ring slots
   int chunk_pieces;       // 16-byte pieces per chunk (per array)
   int per_rank_pieces;    // pieces per slice (last rank may own fewer)
   int num_clusters;
@@ -63,16 +73,17 @@ struct StagedPlan {
 };
 
 struct __align__(16) Ctrl {
-  unsigned long long full[kMaxSlots];
-  unsigned long long empty[kMaxSlots];
-  unsigned long long xbar[2];    // sweep-1 records of a row are in (count cl*ns1)
-  unsigned long long qbar[2];    // rank 0 only: squared-norm shares of a row are in (count cl*ns2)
-  unsigned long long sbar;       // fallback records are in (count cl*ns2)
+  unsigned long long res_full[kMaxRes];
+  unsigned long long res_empty[kMaxRes];
+  unsigned long long ring_full[kMaxRing];
+  unsigned long long ring_empty[kMaxRing];
+  unsigned long long xbar[2];
+  unsigned long long sbar;
   int abort_flag;
   int pad;
-  float xbuf[2][kMaxRec1][8];    // per row parity: one record per (rank, sweep-1 warp)
-  float sbuf[2][kMaxRec2][8];    // records of the running-maximum fallback, by round parity
-  float qbuf[2][kMaxRec2];       // rank 0 only
+  float xbuf[2][kMaxRec][8];   // per row parity: one record per (rank, warp)
+  float sbuf[kMaxRec][8];      // records of the running-maximum fallback
+  int16_t tab[kMaxChunks];     // chunk j -> resident slot k (>= 0) or -1 (streamed)
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
@@ -169,6 +180,39 @@ __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, vola
     }
   }
 }
+
+// Walks the compact list of processed rows.  The prefix sums of the current sequence are cached
+// in registers, so locating a row touches global memory only when it crosses into a new sequence.
+struct RowCursor {
+  int64_t b, lo, hi;   // sequence, offsets[b], offsets[b+1]
+  int32_t ew;          // effective window of sequence b
+  __device__ __forceinline__ void init(const KlParams& p) {
+    b = 0;
+    lo = 0;
+    hi = p.B > 0 ? p.offsets[1] : 0;
+    ew = p.B > 0 ? p.ewin[0] : 0;
+  }
+  // Global row of processed-row ordinal n (ordinals must not decrease) and whether its gradient
+  // is written.
+  __device__ __forceinline__ int64_t locate(const KlParams& p, int64_t n, bool& wg) {
+    while (n >= hi && b + 1 < p.B) {
+      ++b;
+      lo = hi;
+      hi = p.offsets[b + 1];
+      ew = p.ewin[b];
+    }
+    const int64_t t = n - lo;
+    wg = (p.grad != nullptr) && (t < ew);
+    return b * p.T + t;
+  }
+  __device__ __forceinline__ void fetch_row(const KlParams& p, int64_t ordinal, bool in_range,
+                                            int64_t& r, int& y, bool& wg) {
+    if (in_range) {
+      r = locate(p, ordinal, wg);
+      y = p.tokens[r];
+    }
+  }
+};
 
 // ---------------------------------------------------------------------------- packed fp32 pairs
 // sm_100 issues add/mul/fma on two fp32 lanes held in a 64-bit register pair in one slot
@@ -302,6 +346,7 @@ __device__ __forceinline__ void store_pairs(char* dst, const f2_t (&G)[NP]) {
   }
 }
 
+// The two logits at the sampled token (at element 0 when the token is out of range).
 template <typename TIn>
 __device__ __forceinline__ void fetch_logits_at(const KlParams& p, int64_t r, int y, float& zy,
                                                 float& uy) {
@@ -311,81 +356,12 @@ __device__ __forceinline__ void fetch_logits_at(const KlParams& p, int64_t r, in
   uy = Elem<TIn>::load1(static_cast<const char*>(p.teacher) + (size_t)r * p.ld * sizeof(TIn), yi);
 }
 
-// Walks the compact list of processed rows.  The prefix sums of the current sequence are cached
-// in registers, so locating a row touches global memory only when it crosses into a new sequence.
-struct RowCursor {
-  int64_t b, lo, hi;   // sequence, offsets[b], offsets[b+1]
-  int32_t ew;          // effective window of sequence b
-  __device__ __forceinline__ void init(const KlParams& p) {
-    b = 0;
-    lo = 0;
-    hi = p.B > 0 ? p.offsets[1] : 0;
-    ew = p.B > 0 ? p.ewin[0] : 0;
-  }
-  // Global row of processed-row ordinal n (ordinals must not decrease) and whether its gradient
-  // is written.
-  __device__ __forceinline__ int64_t locate(const KlParams& p, int64_t n, bool& wg) {
-    while (n >= hi && b + 1 < p.B) {
-      ++b;
-      lo = hi;
-      hi = p.offsets[b + 1];
-      ew = p.ewin[b];
-    }
-    const int64_t t = n - lo;
-    wg = (p.grad != nullptr) && (t < ew);
-    return b * p.T + t;
-  }
-};
-
-// Row metadata pipeline of one role: the current row (C) and the next one (N) in registers; the
-// token of row i+2 and the logits at the token of row i+1 are requested while row i is processed.
-template <typename TIn>
-struct RowPipe {
-  RowCursor cur;
-  int64_t rC, rN;
-  int yC, yN;
-  float zyC, uyC;
-  bool wgC, wgN;
-  int64_t rNN;
-  int yNN;
-  float zyN, uyN;
-  bool wgNN;
-  int64_t base, step, count;
-  __device__ __forceinline__ void fetch_row(const KlParams& p, int64_t i, int64_t& r, int& y,
-                                            bool& wg) {
-    if (i < count) {
-      r = cur.locate(p, base + i * step, wg);
-      y = p.tokens[r];
-    }
-  }
-  __device__ __forceinline__ void init(const KlParams& p, int64_t base_, int64_t step_,
-                                       int64_t count_) {
-    base = base_;
-    step = step_;
-    count = count_;
-    cur.init(p);
-    rC = rN = 0;
-    yC = yN = 0;
-    zyC = uyC = 0.f;
-    wgC = wgN = false;
-    fetch_row(p, 0, rC, yC, wgC);
-    if (count > 0) fetch_logits_at<TIn>(p, rC, yC, zyC, uyC);
-    fetch_row(p, 1, rN, yN, wgN);
-  }
-  // At the top of iteration i: request what iterations i+1 and i+2 will need.
-  __device__ __forceinline__ void prefetch(const KlParams& p, int64_t i) {
-    zyN = uyN = 0.f;
-    rNN = 0;
-    yNN = 0;
-    wgNN = false;
-    if (i + 1 < count) fetch_logits_at<TIn>(p, rN, yN, zyN, uyN);
-    fetch_row(p, i + 2, rNN, yNN, wgNN);
-  }
-  __device__ __forceinline__ void rotate() {
-    rC = rN; yC = yN; wgC = wgN; zyC = zyN; uyC = uyN;
-    rN = rNN; yN = yNN; wgN = wgNN;
-  }
-};
+// Chunk j of a slice is resident iff the running count floor(j*nres/nch) steps at j: the nres
+// resident chunks are spread evenly along the slice.  Returns the resident slot or -1.
+__device__ __forceinline__ int resident_slot(int j, int nres, int nch) {
+  const int a = (j * nres) / nch, b = ((j + 1) * nres) / nch;
+  return b > a ? a : -1;
+}
 
 // Fixed-order sum over the lanes of a warp; every lane returns the same bits.
 __device__ __forceinline__ float lane_sum(float v) {
@@ -400,15 +376,15 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
   constexpr int NP = Pairs<TIn>::NP;
   extern __shared__ __align__(128) char smem[];
   Ctrl& ctrl = *reinterpret_cast<Ctrl*>(smem);
-  char* ring = smem + kCtrlBytes;
+  char* res_base = smem + kCtrlBytes;
+  char* ring_base = res_base + (size_t)plan.nres * plan.slot_bytes;
   volatile int* abort = &ctrl.abort_flag;
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_rank();
   const int cl = plan.cl;
-  const int ns1 = plan.ns1, ns2 = plan.ns2;
-  const int nch = plan.nch, nslot = plan.nslot;
+  const int nch = plan.nch, nres = plan.nres, nring = plan.nring;
   const int64_t cluster_id = blockIdx.x / cl;
   const uint32_t u_off = (uint32_t)plan.chunk_pieces * 16u;
 
@@ -423,15 +399,18 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       cluster_id < total_rows ? (total_rows - cluster_id + plan.num_clusters - 1) / plan.num_clusters : 0;
 
   if (tid == 0) {
-    for (int s = 0; s < nslot; ++s) {
-      mbar_init(smem_u32(&ctrl.full[s]), 1);
-      mbar_init(smem_u32(&ctrl.empty[s]), kNC);
+    for (int s = 0; s < nres; ++s) {
+      mbar_init(smem_u32(&ctrl.res_full[s]), 1);
+      mbar_init(smem_u32(&ctrl.res_empty[s]), kGW);
     }
-    for (int k = 0; k < 2; ++k) {
-      mbar_init(smem_u32(&ctrl.xbar[k]), cl * ns1);
-      mbar_init(smem_u32(&ctrl.qbar[k]), cl * ns2);
+    for (int s = 0; s < nring; ++s) {
+      mbar_init(smem_u32(&ctrl.ring_full[s]), 1);
+      mbar_init(smem_u32(&ctrl.ring_empty[s]), kNW);
     }
-    mbar_init(smem_u32(&ctrl.sbar), cl * ns2);
+    for (int j = 0; j < nch; ++j) ctrl.tab[j] = (int16_t)resident_slot(j, nres, nch);
+    mbar_init(smem_u32(&ctrl.xbar[0]), cl * kNW);
+    mbar_init(smem_u32(&ctrl.xbar[1]), cl * kNW);
+    mbar_init(smem_u32(&ctrl.sbar), cl * kNW);
     ctrl.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -443,11 +422,29 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
     const int left = (int)my_pieces - j * plan.chunk_pieces;
     return left < plan.chunk_pieces ? left : plan.chunk_pieces;
   };
-  bool timed_out = false;
+  // issue the two bulk copies of chunk j of row r into a slot
+  auto issue_chunk = [&](int64_t r, int j, char* slot, unsigned long long* full) {
+    int np = pieces_in_chunk(j);
+    np = np < 0 ? 0 : np;
+    const uint32_t bytes = (uint32_t)np * 16u;
+    const uint32_t bar = smem_u32(full);
+    if (bytes == 0) {
+      mbar_arrive(bar);
+    } else {
+      const size_t goff = ((size_t)r * p.ld + (size_t)piece0 * N) * sizeof(TIn) +
+                          (size_t)j * plan.chunk_pieces * 16;
+      mbar_arrive_expect_tx(bar, 2u * bytes);
+      const uint32_t dst = smem_u32(slot);
+      bulk_load(dst, static_cast<const char*>(p.student) + goff, bytes, bar);
+      bulk_load(dst + u_off, static_cast<const char*>(p.teacher) + goff, bytes, bar);
+    }
+  };
 
-  if (warp == kProducerWarp) {
-    // ------------------------------------------------------------------ producer lane
-    if (lane == 0) {
+  if (warp == kProducerWarp && lane == 0) {
+    // ------------------------------------------------------------------ ring producer
+    // Order of the stream: per row, the streamed chunks for sweep 1, then (rows whose gradient is
+    // written) the same chunks again for sweep 2.
+    if (nring > 0 && nres < nch) {
       int slot = 0;
       uint32_t phase = 0;
       int64_t fills = 0;
@@ -455,46 +452,35 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       cur.init(p);
       bool stop = false;
       for (int64_t i = 0; i < my_rows && !stop && !*abort; ++i) {
-        bool wg_unused;
-        const int64_t r = cur.locate(p, cluster_id + i * plan.num_clusters, wg_unused);
-        const size_t row_off = ((size_t)r * p.ld + (size_t)piece0 * N) * sizeof(TIn);
-        for (int j = 0; j < nch; ++j) {
-          if (fills >= nslot &&
-              !bounded_wait<false>(smem_u32(&ctrl.empty[slot]), phase ^ 1u, abort)) {
-            stop = true;   // gave up: never overwrite a slot that may still be read
-            break;
-          }
-          int np = pieces_in_chunk(j);
-          np = np < 0 ? 0 : np;
-          const uint32_t bytes = (uint32_t)np * 16u;
-          const uint32_t bar = smem_u32(&ctrl.full[slot]);
-          if (bytes == 0) {
-            mbar_arrive(bar);
-          } else {
-            const size_t goff = row_off + (size_t)j * plan.chunk_pieces * 16;
-            mbar_arrive_expect_tx(bar, 2u * bytes);
-            const uint32_t dst = smem_u32(ring + (size_t)slot * plan.slot_bytes);
-            bulk_load(dst, static_cast<const char*>(p.student) + goff, bytes, bar);
-            bulk_load(dst + u_off, static_cast<const char*>(p.teacher) + goff, bytes, bar);
-          }
-          ++fills;
-          if (++slot == nslot) {
-            slot = 0;
-            phase ^= 1u;
+        bool wg;
+        const int64_t r = cur.locate(p, cluster_id + i * plan.num_clusters, wg);
+        for (int sweep = 0; sweep < (wg ? 2 : 1) && !stop; ++sweep) {
+          for (int j = 0; j < nch; ++j) {
+            if (ctrl.tab[j] >= 0) continue;
+            if (fills >= nring &&
+                !bounded_wait<false>(smem_u32(&ctrl.ring_empty[slot]), phase ^ 1u, abort)) {
+              stop = true;   // gave up: never overwrite a slot that may still be read
+              break;
+            }
+            issue_chunk(r, j, ring_base + (size_t)slot * plan.slot_bytes, &ctrl.ring_full[slot]);
+            ++fills;
+            if (++slot == nring) {
+              slot = 0;
+              phase ^= 1u;
+            }
           }
         }
       }
       // Drain: every copy this CTA issued must have landed before its shared memory goes away.
-      // Walk back over the last min(fills, nslot) fills.
-      int64_t pending = fills < nslot ? fills : nslot;
+      int64_t pending = fills < nring ? fills : nring;
       const uint64_t t0 = global_timer();
       bool gave_up = false;
       while (pending > 0) {
         if (--slot < 0) {
-          slot = nslot - 1;
+          slot = nring - 1;
           phase ^= 1u;
         }
-        const uint32_t bar = smem_u32(&ctrl.full[slot]);
+        const uint32_t bar = smem_u32(&ctrl.ring_full[slot]);
         while (!gave_up && !mbar_try_wait(bar, phase)) {
           if (global_timer() - t0 > kWaitLimitNs) gave_up = true;
         }
@@ -502,153 +488,178 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       }
       if (gave_up) atomicOr(p.status, ADWIN_DEV_TIMEOUT);
     }
-  } else if (warp < ns1) {
-    // ------------------------------------------------------------------ sweep-1 warps
-    const int t1 = ns1 * 32;                      // threads of this role
-    const uint32_t toff = (uint32_t)tid * 16u;    // first of this thread's kP1 pieces in a chunk
-    int slot = 0;
-    uint32_t phase = 0;
-    RowPipe<TIn> rp;
-    rp.init(p, cluster_id, plan.num_clusters, my_rows);
-    for (int64_t i = 0; i < my_rows; ++i) {
-      rp.prefetch(p, i);
-      const bool wg = rp.wgC;
-      const float ref_s = rp.zyC * kLog2e, ref_t = rp.uyC * kLog2e;   // shared references
-      const float dref = wg ? 0.f : rp.zyC - rp.uyC;                  // delta is centred on probe rows
-      const f2_t nrefs = splat2(-ref_s), nreft = splat2(-ref_t), ndref = splat2(-dref);
-      Acc2 a;
-      a.reset();
-      for (int j = 0; j < nch; ++j) {
-        if (!bounded_wait<false>(smem_u32(&ctrl.full[slot]), phase, abort)) {
-          timed_out = true;
-          break;
-        }
-        // The thread's pieces go to registers and the warp is done with the slot at once.
-        const char* sl = ring + (size_t)slot * plan.slot_bytes + toff;
-        const int np = pieces_in_chunk(j);
-        uint4 zr[kP1], ur[kP1];
-#pragma unroll
-        for (int h = 0; h < kP1; ++h) {
-          if (tid + h * t1 < np) {
-            zr[h] = *reinterpret_cast<const uint4*>(sl + (size_t)h * t1 * 16);
-            ur[h] = *reinterpret_cast<const uint4*>(sl + u_off + (size_t)h * t1 * 16);
-          }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&ctrl.empty[slot]));
-#pragma unroll
-        for (int h = 0; h < kP1; ++h) {
-          if (tid + h * t1 < np) {
-            f2_t Z[NP], U[NP];
-            Pairs<TIn>::make(zr[h], Z);
-            Pairs<TIn>::make(ur[h], U);
-            if (wg)
-              acc_grad<NP>(Z, U, nrefs, nreft, a);
-            else
-              acc_probe<NP>(Z, U, nrefs, nreft, ndref, a);
-          }
-        }
-        if (++slot == nslot) {
-          slot = 0;
-          phase ^= 1u;
+  } else if (warp == kProducerWarp && lane == 1) {
+    // ------------------------------------------------------------------ resident producer
+    // Resident slot k takes resident chunk k of every row: fill number i belongs to row i and
+    // waits for drain number i-1 (sweep 2 of row i-1, or its sweep 1 if no gradient is written).
+    if (nres > 0) {
+      RowCursor cur;
+      cur.init(p);
+      int64_t last_row = -1;   // last row some slot was filled for, and how many slots got it
+      int last_k = 0;
+      for (int64_t i = 0; i < my_rows && !*abort; ++i) {
+        bool wg_unused;
+        const int64_t r = cur.locate(p, cluster_id + i * plan.num_clusters, wg_unused);
+        for (int j = 0; j < nch; ++j) {
+          const int k = ctrl.tab[j];
+          if (k < 0) continue;
+          if (i > 0 &&
+              !bounded_wait<false>(smem_u32(&ctrl.res_empty[k]), (uint32_t)((i - 1) & 1), abort))
+            break;   // gave up: never overwrite a slot that may still be read
+          issue_chunk(r, j, res_base + (size_t)k * plan.slot_bytes, &ctrl.res_full[k]);
+          last_row = i;
+          last_k = k + 1;
         }
       }
-      if (timed_out) break;
-      // record = { S, A, St, B0, B1, B2, 0, 0 }: this warp's sums over its lanes, to every CTA
-      const float v0 = lane_sum(hsum2(a.S)), v1 = lane_sum(hsum2(a.A)), v2 = lane_sum(hsum2(a.St));
-      float v3 = 0.f, v4 = 0.f, v5 = 0.f;
-      if (!wg) {
-        v3 = lane_sum(hsum2(a.B0));
-        v4 = lane_sum(hsum2(a.B1));
-        v5 = lane_sum(hsum2(a.B2));
+      // Drain: the last fill of every resident slot must have landed before the CTA exits
+      // (slots k < last_k were filled for last_row, the others for the row before).
+      const uint64_t t0 = global_timer();
+      bool gave_up = false;
+      for (int k = 0; k < nres; ++k) {
+        const int64_t fill = k < last_k ? last_row : last_row - 1;
+        if (fill < 0) continue;
+        const uint32_t bar = smem_u32(&ctrl.res_full[k]);
+        while (!gave_up && !mbar_try_wait(bar, (uint32_t)(fill & 1))) {
+          if (global_timer() - t0 > kWaitLimitNs) gave_up = true;
+        }
       }
-      const int par = (int)(i & 1);
-      if (lane < cl) {
-        const uint32_t dst =
-            map_to_rank(smem_u32(&ctrl.xbuf[par][rank * ns1 + warp][0]), (uint32_t)lane);
-        remote_store4(dst, v0, v1, v2, v3);
-        remote_store4(dst + 16, v4, v5, 0.f, 0.f);
-        remote_arrive_release(map_to_rank(smem_u32(&ctrl.xbar[par]), (uint32_t)lane));
-      }
-      rp.rotate();
+      if (gave_up) atomicOr(p.status, ADWIN_DEV_TIMEOUT);
     }
-  } else {
-    // ------------------------------------------------------------------ sweep-2 warps
+  } else if (warp < kNW) {
+    // ------------------------------------------------------------------ consumer warps
     const bool full_mode = (p.mode == ADWIN_GRAD_FULL_KL);
-    const int w2 = warp - ns1;                    // warp index inside the role
-    const int g2 = tid - ns1 * 32;                // thread index inside the role
-    const int t2 = ns2 * 32;
-    const int nrec1 = cl * ns1, nrec2 = cl * ns2;
-    const uint32_t toff = (uint32_t)g2 * 16u;
-    int slot = 0;
-    uint32_t phase = 0;
+    const int nrec = cl * kNW;
+    int rc_slot = 0;            // ring cursor
+    uint32_t rc_phase = 0;
     uint32_t safe_rounds = 0;   // completed fallback exchanges (parity of sbar)
+    bool timed_out = false;
+    float q_prev = 0.f;         // this warp's share of the previous written row's squared norm
     int64_t r_prev = 0;
     bool wg_prev = false;
-    RowPipe<TIn> rp;
-    rp.init(p, cluster_id, plan.num_clusters, my_rows);
 
-    // rank 0, first sweep-2 warp: the squared norm of a written gradient row, once every
-    // sweep-2 warp of the cluster has delivered its share
-    auto collect_norm = [&](int64_t i_prev) -> bool {
-      if (rank != 0 || w2 != 0) return true;
-      const int par = (int)(i_prev & 1);
-      if (!bounded_wait<true>(smem_u32(&ctrl.qbar[par]), (uint32_t)((i_prev >> 1) & 1), abort))
-        return false;
-      float s = 0.f;
-      for (int rr = lane; rr < nrec2; rr += 32) s += ctrl.qbuf[par][rr];
-      s = lane_sum(s);
-      if (lane == 0 && wg_prev && p.gsq) p.gsq[r_prev] = s;
-      return true;
-    };
+    // metadata pipeline: current row (C) and next row (N) held in registers
+    RowCursor cur;
+    cur.init(p);
+    int64_t rC = 0, rN = 0;
+    int yC = 0, yN = 0;
+    float zyC = 0.f, uyC = 0.f;
+    bool wgC = false, wgN = false;
+    cur.fetch_row(p, cluster_id, 0 < my_rows, rC, yC, wgC);
+    if (my_rows > 0) fetch_logits_at<TIn>(p, rC, yC, zyC, uyC);
+    cur.fetch_row(p, cluster_id + plan.num_clusters, 1 < my_rows, rN, yN, wgN);
 
-    for (int64_t i = 0; i < my_rows; ++i) {
-      rp.prefetch(p, i);
-      const bool wg = rp.wgC;
-      const int64_t r = rp.rC;
-      const int y = rp.yC;
-      const float zy = rp.zyC, uy = rp.uyC;
-      const bool y_valid = (y >= 0) && ((int64_t)y < p.V);
-      const float ref_s = zy * kLog2e, ref_t = uy * kLog2e;
-      const float dref = wg ? 0.f : zy - uy;
-      const int par = (int)(i & 1);
+    const int grp = warp / kGW;                  // this warp's group: chunks j % kG == grp
+    const int gt = tid - grp * kGT;              // thread index inside the group
+    const uint32_t toff = (uint32_t)gt * 16u;    // first of this thread's kP pieces in a chunk
+    const int64_t iters = my_rows > 0 ? my_rows + 1 : 0;   // + one exchange for the last norm
+    for (int64_t i = 0; i < iters; ++i) {
+      const bool real = i < my_rows;
+      // next rows' dependent loads, consumed one iteration later
+      float zyN = 0.f, uyN = 0.f;
+      int64_t rNN = 0;
+      int yNN = 0;
+      bool wgNN = false;
+      if (i + 1 < my_rows) fetch_logits_at<TIn>(p, rN, yN, zyN, uyN);
+      cur.fetch_row(p, cluster_id + (i + 2) * plan.num_clusters, i + 2 < my_rows, rNN, yNN, wgNN);
 
-      // Before this warp releases anything of row i: the two-deep norm buffer of row i-1 is read.
-      if (i > 0 && !collect_norm(i - 1)) {
-        timed_out = true;
-        break;
-      }
-      if (!wg) {
-        // Row without a gradient: sweep 2 has nothing to read, but every consumer warp observes
-        // and releases every fill of a slot, and it does so as the chunks land, not after the
-        // row's totals, so that such rows stream through a ring smaller than a row.
+      const bool y_valid = (yC >= 0) && ((int64_t)yC < p.V);
+      const float ref_s = zyC * kLog2e, ref_t = uyC * kLog2e;   // shared references of the row
+      const float dref = wgC ? 0.f : zyC - uyC;                 // delta is centred on probe rows
+      const uint32_t rpar = (uint32_t)(i & 1);                  // fill parity of resident slots
+
+      // ---------------------------------------------------------------- sweep 1
+      Acc2 a;
+      a.reset();
+      if (real) {
+        const f2_t nrefs = splat2(-ref_s), nreft = splat2(-ref_t), ndref = splat2(-dref);
         for (int j = 0; j < nch; ++j) {
-          if (!bounded_wait<false>(smem_u32(&ctrl.full[slot]), phase, abort)) {
-            timed_out = true;
-            break;
+          const int k = ctrl.tab[j];
+          if (j % kG == grp) {
+            const char* sl;
+            if (k >= 0) {
+              if (!bounded_wait<false>(smem_u32(&ctrl.res_full[k]), rpar, abort)) timed_out = true;
+              sl = res_base + (size_t)k * plan.slot_bytes + toff;
+            } else {
+              if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort)) timed_out = true;
+              sl = ring_base + (size_t)rc_slot * plan.slot_bytes + toff;
+            }
+            if (timed_out) break;
+            // The thread's pieces go to registers first and the slot is handed back at once, so
+            // the refill is in flight while the arithmetic runs.
+            const int np = pieces_in_chunk(j);
+            uint4 zr[kP], ur[kP];
+#pragma unroll
+            for (int h = 0; h < kP; ++h) {
+              if (gt + h * kGT < np) {
+                zr[h] = *reinterpret_cast<const uint4*>(sl + h * kGT * 16);
+                ur[h] = *reinterpret_cast<const uint4*>(sl + u_off + h * kGT * 16);
+              }
+            }
+            if (k < 0 || !wgC) {
+              __syncwarp();
+              if (lane == 0)
+                mbar_arrive(smem_u32(k < 0 ? &ctrl.ring_empty[rc_slot] : &ctrl.res_empty[k]));
+            }
+#pragma unroll
+            for (int h = 0; h < kP; ++h) {
+              if (gt + h * kGT < np) {
+                f2_t Z[NP], U[NP];
+                Pairs<TIn>::make(zr[h], Z);
+                Pairs<TIn>::make(ur[h], U);
+                if (wgC)
+                  acc_grad<NP>(Z, U, nrefs, nreft, a);
+                else
+                  acc_probe<NP>(Z, U, nrefs, nreft, ndref, a);
+              }
+            }
+          } else if (k < 0) {
+            // Not this group's chunk, but every warp observes and releases every fill of a ring
+            // slot: a parity wait is only sound within one phase of the barrier's current one.
+            if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort)) {
+              timed_out = true;
+              break;
+            }
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl.ring_empty[rc_slot]));
           }
-          if (lane == 0) mbar_arrive(smem_u32(&ctrl.empty[slot]));
-          if (++slot == nslot) {
-            slot = 0;
-            phase ^= 1u;
+          if (k < 0 && ++rc_slot == nring) {   // the ring cursor walks every streamed chunk
+            rc_slot = 0;
+            rc_phase ^= 1u;
           }
         }
         if (timed_out) break;
       }
 
-      // ---------------------------------------------------------------- totals of row i
-      if (!bounded_wait<true>(smem_u32(&ctrl.xbar[par]), (uint32_t)((i >> 1) & 1), abort)) {
-        timed_out = true;
-        break;
-      }
+      // ---------------------------------------------------------------- exchange
+      // record = { S, A, St, B0, B1, B2, q_prev, 0 }: this warp's sums over its lanes.
       RowTotals t;
+      float qtot;
       {
-        float s[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        for (int rr = lane; rr < nrec1; rr += 32) {
+        const float v0 = lane_sum(hsum2(a.S)), v1 = lane_sum(hsum2(a.A)), v2 = lane_sum(hsum2(a.St));
+        float v3 = 0.f, v4 = 0.f, v5 = 0.f;
+        if (real && !wgC) {
+          v3 = lane_sum(hsum2(a.B0));
+          v4 = lane_sum(hsum2(a.B1));
+          v5 = lane_sum(hsum2(a.B2));
+        }
+        const int par = (int)(i & 1);
+        if (lane < cl) {
+          const uint32_t dst =
+              map_to_rank(smem_u32(&ctrl.xbuf[par][rank * kNW + warp][0]), (uint32_t)lane);
+          remote_store4(dst, v0, v1, v2, v3);
+          remote_store4(dst + 16, v4, v5, q_prev, 0.f);
+          remote_arrive_release(map_to_rank(smem_u32(&ctrl.xbar[par]), (uint32_t)lane));
+        }
+        if (!bounded_wait<true>(smem_u32(&ctrl.xbar[par]), (uint32_t)((i >> 1) & 1), abort)) {
+          timed_out = true;
+          break;
+        }
+        // fixed-order sum of the nrec records (lane = record, then a butterfly)
+        float s[7] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int rr = lane; rr < nrec; rr += 32) {
           const float4 x0 = *reinterpret_cast<const float4*>(&ctrl.xbuf[par][rr][0]);
           const float4 x1 = *reinterpret_cast<const float4*>(&ctrl.xbuf[par][rr][4]);
           s[0] += x0.x; s[1] += x0.y; s[2] += x0.z; s[3] += x0.w;
-          s[4] += x1.x; s[5] += x1.y;
+          s[4] += x1.x; s[5] += x1.y; s[6] += x1.z;
         }
         t.M2s = ref_s;
         t.M2t = ref_t;
@@ -656,77 +667,58 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
         t.A = lane_sum(s[1]);
         t.St = lane_sum(s[2]);
         t.B0 = t.B1 = t.B2 = 0.f;
-        if (!wg) {
+        if (real && !wgC) {
           t.B0 = lane_sum(s[3]);
           t.B1 = lane_sum(s[4]);
           t.B2 = lane_sum(s[5]);
         }
+        qtot = lane_sum(s[6]);
       }
+      if (warp == 0 && lane == 0 && rank == 0 && i > 0 && wg_prev && p.gsq) p.gsq[r_prev] = qtot;
+      if (!real) break;
+
       // ---------------------------------------------------------------- overflow fallback
-      // The totals are identical in every sweep-2 warp of the cluster, so this branch is uniform.
+      // The totals are identical in every warp of the cluster, so this branch is uniform.
       if (!(t.S < kSumLimit) || !(t.St < kSumLimit) || !(t.B0 < kSumLimit)) {
-        // Few threads share a long slice here, so the running sums are kept in double and fed in
-        // blocks of 8 pieces (each block accumulated in fp32 against its own running maximum).
-        const char* zrow = static_cast<const char*>(p.student) + ((size_t)r * p.ld + (size_t)piece0 * N) * sizeof(TIn);
-        const char* urow = static_cast<const char*>(p.teacher) + ((size_t)r * p.ld + (size_t)piece0 * N) * sizeof(TIn);
-        double dS = 0.0, dA = 0.0, dB0 = 0.0, dB1 = 0.0, dB2 = 0.0, dSt = 0.0;
-        float Ms = -INFINITY, Mt = -INFINITY;
-        for (int64_t pc0 = g2; pc0 < my_pieces; pc0 += (int64_t)8 * t2) {
-          RowAcc ra;
-          ra.reset();
-          for (int b8 = 0; b8 < 8; ++b8) {
-            const int64_t pc = pc0 + (int64_t)b8 * t2;
-            if (pc >= my_pieces) break;
-            float z[N], u[N];
-            const uint4 zv = __ldg(reinterpret_cast<const uint4*>(zrow) + pc);
-            const uint4 uv = __ldg(reinterpret_cast<const uint4*>(urow) + pc);
-            Elem<TIn>::unpack(zv, z);
-            Elem<TIn>::unpack(uv, u);
-            acc_piece<N, true>(z, u, dref, ra);
-          }
-          const float nMs = fmaxf(Ms, ra.m2s), nMt = fmaxf(Mt, ra.m2t);
-          const double fo = (Ms == -INFINITY) ? 0.0 : exp2((double)(Ms - nMs));
-          const double fn = (ra.m2s == -INFINITY) ? 0.0 : exp2((double)(ra.m2s - nMs));
-          const double go = (Mt == -INFINITY) ? 0.0 : exp2((double)(Mt - nMt));
-          const double gn = (ra.m2t == -INFINITY) ? 0.0 : exp2((double)(ra.m2t - nMt));
-          dS = dS * fo + (double)ra.S * fn;
-          dA = dA * fo + (double)ra.A * fn;
-          dB0 = dB0 * (fo * fo) + (double)ra.B0 * (fn * fn);
-          dB1 = dB1 * (fo * fo) + (double)ra.B1 * (fn * fn);
-          dB2 = dB2 * (fo * fo) + (double)ra.B2 * (fn * fn);
-          dSt = dSt * go + (double)ra.St * gn;
-          Ms = nMs;
-          Mt = nMt;
+        RowAcc ra;
+        ra.reset();
+        const char* zrow = static_cast<const char*>(p.student) + ((size_t)rC * p.ld + (size_t)piece0 * N) * sizeof(TIn);
+        const char* urow = static_cast<const char*>(p.teacher) + ((size_t)rC * p.ld + (size_t)piece0 * N) * sizeof(TIn);
+        for (int64_t pc = tid; pc < my_pieces; pc += kNT) {
+          float z[N], u[N];
+          const uint4 zv = __ldg(reinterpret_cast<const uint4*>(zrow) + pc);
+          const uint4 uv = __ldg(reinterpret_cast<const uint4*>(urow) + pc);
+          Elem<TIn>::unpack(zv, z);
+          Elem<TIn>::unpack(uv, u);
+          acc_piece<N, true>(z, u, dref, ra);
         }
-        const float wms = warp_max(Ms), wmt = warp_max(Mt);
-        const double fs = (Ms == -INFINITY) ? 0.0 : exp2((double)(Ms - wms));
-        const double ft = (Mt == -INFINITY) ? 0.0 : exp2((double)(Mt - wmt));
-        const float x1 = lane_sum((float)(dS * fs)), x2 = lane_sum((float)(dA * fs));
-        const float x3 = lane_sum((float)(dB0 * fs * fs)), x4 = lane_sum((float)(dB1 * fs * fs));
-        const float x5 = lane_sum((float)(dB2 * fs * fs)), x7 = lane_sum((float)(dSt * ft));
+        const float wms = warp_max(ra.m2s), wmt = warp_max(ra.m2t);
+        const float fs = (ra.m2s == -INFINITY) ? 0.f : ex2f(ra.m2s - wms);
+        const float ft = (ra.m2t == -INFINITY) ? 0.f : ex2f(ra.m2t - wmt);
+        const float fs2 = fs * fs;
+        const float w1 = lane_sum(ra.S * fs), w2 = lane_sum(ra.A * fs), w3 = lane_sum(ra.B0 * fs2);
+        const float w4 = lane_sum(ra.B1 * fs2), w5 = lane_sum(ra.B2 * fs2), w7 = lane_sum(ra.St * ft);
         if (lane < cl) {
-          const uint32_t dst =
-              map_to_rank(smem_u32(&ctrl.sbuf[safe_rounds & 1u][rank * ns2 + w2][0]), (uint32_t)lane);
-          remote_store4(dst, wms, x1, x2, x3);
-          remote_store4(dst + 16, x4, x5, wmt, x7);
+          const uint32_t dst = map_to_rank(smem_u32(&ctrl.sbuf[rank * kNW + warp][0]), (uint32_t)lane);
+          remote_store4(dst, wms, w1, w2, w3);
+          remote_store4(dst + 16, w4, w5, wmt, w7);
           remote_arrive_release(map_to_rank(smem_u32(&ctrl.sbar), (uint32_t)lane));
         }
         if (!bounded_wait<true>(smem_u32(&ctrl.sbar), safe_rounds & 1u, abort)) {
           timed_out = true;
           break;
         }
-        const float(*sb)[8] = ctrl.sbuf[safe_rounds & 1u];
         ++safe_rounds;
         float ms = -INFINITY, mt = -INFINITY;
-        for (int rr = lane; rr < nrec2; rr += 32) {
-          ms = fmaxf(ms, sb[rr][0]);
-          mt = fmaxf(mt, sb[rr][6]);
+        for (int rr = lane; rr < nrec; rr += 32) {
+          ms = fmaxf(ms, ctrl.sbuf[rr][0]);
+          mt = fmaxf(mt, ctrl.sbuf[rr][6]);
         }
         t.M2s = warp_max(ms);
         t.M2t = warp_max(mt);
         float s[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        for (int rr = lane; rr < nrec2; rr += 32) {
-          const float* x = sb[rr];
+        for (int rr = lane; rr < nrec; rr += 32) {
+          const float* x = ctrl.sbuf[rr];
           const float gs = (x[0] == -INFINITY) ? 0.f : ex2f(x[0] - t.M2s);
           const float gt = (x[6] == -INFINITY) ? 0.f : ex2f(x[6] - t.M2t);
           const float gs2 = gs * gs;
@@ -739,18 +731,16 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
         t.B1 = lane_sum(s[3]);
         t.B2 = lane_sum(s[4]);
         t.St = lane_sum(s[5]);
-        // Round k+2 reuses the buffer of round k; it cannot start before round k+1 is complete,
-        // which needs an arrival from every warp, made after it has read round k.
       }
 
       // ---------------------------------------------------------------- row scalars
-      const RowScalars rs = finish_row(t, zy, uy, y_valid, dref, p.alpha, p.mode);
-      if (w2 == 0 && lane == 0 && rank == 0) {
-        p.kl[r] = rs.kl;
-        p.logratio[r] = rs.c;
-        if (p.gsq && !wg) p.gsq[r] = rs.gsq_expanded;
-        if (p.lse_s) p.lse_s[r] = rs.lse_s;
-        if (p.lse_t) p.lse_t[r] = rs.lse_t;
+      const RowScalars rs = finish_row(t, zyC, uyC, y_valid, dref, p.alpha, p.mode);
+      if (warp == 0 && lane == 0 && rank == 0) {
+        p.kl[rC] = rs.kl;
+        p.logratio[rC] = rs.c;
+        if (p.gsq && !wgC) p.gsq[rC] = rs.gsq_expanded;
+        if (p.lse_s) p.lse_s[rC] = rs.lse_s;
+        if (p.lse_t) p.lse_t[rC] = rs.lse_t;
         int bits = 0;
         if (!y_valid) bits |= ADWIN_DEV_TOKEN_RANGE;
         if (rs.nonfinite) bits |= ADWIN_DEV_NONFINITE;
@@ -758,42 +748,41 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       }
 
       // ---------------------------------------------------------------- sweep 2
-      float q = 0.f;
-      if (wg) {
+      q_prev = 0.f;
+      if (wgC) {
         const f2_t L2 = splat2(kLog2e), NEG1 = splat2(-1.f);
         const f2_t nM2s = splat2(-t.M2s), nc0 = splat2(-rs.c0), coef2 = splat2(rs.coef);
-        const int64_t ypiece = y_valid ? ((int64_t)y / N - piece0) : -1;   // slice-relative
+        const int64_t ypiece = y_valid ? ((int64_t)yC / N - piece0) : -1;   // slice-relative
         char* gthread = static_cast<char*>(p.grad) +
-                        ((size_t)r * p.ld_grad + (size_t)(piece0 + g2) * N) * sizeof(TOut);
+                        ((size_t)rC * p.ld_grad + (size_t)(piece0 + gt) * N) * sizeof(TOut);
         const size_t gstep = (size_t)plan.chunk_pieces * N * sizeof(TOut);
         f2_t Q = 0ull;
         for (int j = 0; j < nch; ++j) {
-          if (!bounded_wait<false>(smem_u32(&ctrl.full[slot]), phase, abort)) {
-            timed_out = true;
-            break;
-          }
-          const char* sl = ring + (size_t)slot * plan.slot_bytes + toff;
-          const int np = pieces_in_chunk(j);
+          const int k = ctrl.tab[j];
+          if (j % kG == grp) {
+            const char* sl;
+            if (k >= 0) {
+              sl = res_base + (size_t)k * plan.slot_bytes + toff;   // still there since sweep 1
+            } else {
+              if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort)) timed_out = true;
+              sl = ring_base + (size_t)rc_slot * plan.slot_bytes + toff;
+            }
+            if (timed_out) break;
+            const int np = pieces_in_chunk(j);
+            uint4 zr[kP], ur[kP];
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            constexpr int H = kP2 / 2;
-            uint4 zr[H], ur[H];
-#pragma unroll
-            for (int h = 0; h < H; ++h) {
-              const int hh = half * H + h;
-              if (g2 + hh * t2 < np) {
-                zr[h] = *reinterpret_cast<const uint4*>(sl + (size_t)hh * t2 * 16);
-                ur[h] = *reinterpret_cast<const uint4*>(sl + u_off + (size_t)hh * t2 * 16);
+            for (int h = 0; h < kP; ++h) {
+              if (gt + h * kGT < np) {
+                zr[h] = *reinterpret_cast<const uint4*>(sl + h * kGT * 16);
+                ur[h] = *reinterpret_cast<const uint4*>(sl + u_off + h * kGT * 16);
               }
             }
-            if (half == 1) {   // all pieces of the chunk are in registers: hand the slot back
-              __syncwarp();
-              if (lane == 0) mbar_arrive(smem_u32(&ctrl.empty[slot]));
-            }
+            __syncwarp();
+            if (lane == 0)
+              mbar_arrive(smem_u32(k < 0 ? &ctrl.ring_empty[rc_slot] : &ctrl.res_empty[k]));
 #pragma unroll
-            for (int h = 0; h < H; ++h) {
-              const int hh = half * H + h;
-              if (g2 + hh * t2 < np) {
+            for (int h = 0; h < kP; ++h) {
+              if (gt + h * kGT < np) {
                 f2_t Z[NP], U[NP], G[NP];
                 Pairs<TIn>::make(zr[h], Z);
                 Pairs<TIn>::make(ur[h], U);
@@ -807,8 +796,8 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
                     G[e] = mul2(E, coef2);
                   }
                 }
-                if (!full_mode && (int64_t)j * plan.chunk_pieces + g2 + hh * t2 == ypiece) {
-                  const int e = (int)((int64_t)y - ((int64_t)y / N) * N);
+                if (!full_mode && (int64_t)j * plan.chunk_pieces + gt + h * kGT == ypiece) {
+                  const int e = (int)((int64_t)yC - ((int64_t)yC / N) * N);
 #pragma unroll
                   for (int w = 0; w < NP; ++w) {
                     float lo, hi;
@@ -820,35 +809,37 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
                 }
 #pragma unroll
                 for (int e = 0; e < NP; ++e) Q = fma2(G[e], G[e], Q);
-                store_pairs<TOut, NP>(gthread + (size_t)j * gstep + (size_t)hh * t2 * N * sizeof(TOut), G);
+                store_pairs<TOut, NP>(gthread + (size_t)j * gstep + (size_t)h * kGT * N * sizeof(TOut), G);
               }
             }
+          } else if (k < 0) {
+            if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort)) {
+              timed_out = true;
+              break;
+            }
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl.ring_empty[rc_slot]));
           }
-          if (++slot == nslot) {
-            slot = 0;
-            phase ^= 1u;
+          if (k < 0 && ++rc_slot == nring) {
+            rc_slot = 0;
+            rc_phase ^= 1u;
           }
         }
         if (timed_out) break;
-        q = lane_sum(hsum2(Q));
+        q_prev = lane_sum(hsum2(Q));
       }
-      // this warp's share of the row's squared gradient norm, to rank 0
-      if (lane == 0) {
-        const uint32_t dst = map_to_rank(smem_u32(&ctrl.qbuf[par][rank * ns2 + w2]), 0u);
-        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(dst), "f"(q) : "memory");
-        remote_arrive_release(map_to_rank(smem_u32(&ctrl.qbar[par]), 0u));
-      }
-      r_prev = r;
-      wg_prev = wg;
-      rp.rotate();
+      r_prev = rC;
+      wg_prev = wgC;
+
+      // rotate the metadata pipeline
+      rC = rN; yC = yN; wgC = wgN; zyC = zyN; uyC = uyN;
+      rN = rNN; yN = yNN; wgN = wgNN;
     }
-    if (!timed_out && my_rows > 0 && !collect_norm(my_rows - 1)) timed_out = true;
-  }
-  if (timed_out && lane == 0) {
-    atomicOr(p.status, ADWIN_DEV_TIMEOUT);
-    // let the peers stop waiting as well
-    for (int d = 0; d < cl; ++d)
-      remote_store_u32(map_to_rank(smem_u32(&ctrl.abort_flag), (uint32_t)d), 1u);
+    if (timed_out && lane == 0) {
+      atomicOr(p.status, ADWIN_DEV_TIMEOUT);
+      // let the peers stop waiting as well
+      for (int d = 0; d < cl; ++d)
+        remote_store_u32(map_to_rank(smem_u32(&ctrl.abort_flag), (uint32_t)d), 1u);
+    }
   }
   // No CTA leaves while a peer may still write into its shared memory or arrive on its barriers.
   __syncwarp();
@@ -859,40 +850,42 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
 namespace {
 
 constexpr int kSmemOptin = 232448;   // 227 KB: the per-CTA limit of sm_100
+// Streamed chunks are read a second time by sweep 2; the bytes of one round of rows that have to
+// survive in L2 until then should stay well inside the cache.
+constexpr double kL2BudgetBytes = 32.0 * 1024 * 1024;
 
-// Chunking for one cluster size; false when the ring cannot hold a slice plus two slots.
+// Chunking and the resident / streamed split for one cluster size.
 bool plan_for_cluster(int64_t pieces_total, int cl, bool has_grad, StagedPlan& plan) {
-  const int64_t ring_bytes = kSmemOptin - kCtrlBytes;
+  const int64_t slots_bytes = kSmemOptin - kCtrlBytes;
   const int64_t per_rank = (pieces_total + cl - 1) / cl;
   if (per_rank * 16 > (int64_t)1 << 30) return false;
-  // 10 warps take sweep 1 and 5 take sweep 2 (two exponentials per entry against one); a call
-  // that writes no gradient has no sweep 2 and leaves one warp for the row scalars.
-  const int ns1 = has_grad ? 10 : 14, ns2 = kNC - ns1;
-  int64_t chunk_max = (int64_t)ns1 * 32 * kP1;
-  if (has_grad && (int64_t)ns2 * 32 * kP2 < chunk_max) chunk_max = (int64_t)ns2 * 32 * kP2;
-  int64_t nch = (per_rank + chunk_max - 1) / chunk_max;
-  if (nch < 2 && per_rank >= 16) nch = 2;      // two chunks let consecutive rows overlap
+  int64_t nch = (per_rank + kChunkMax - 1) / kChunkMax;
   int64_t chunk_pieces = (per_rank + nch - 1) / nch;
   chunk_pieces = (chunk_pieces + 7) / 8 * 8;   // slots start on 128-byte boundaries
-  if (chunk_pieces > chunk_max) chunk_pieces = chunk_max;
+  if (chunk_pieces > kChunkMax) chunk_pieces = kChunkMax;
   nch = (per_rank + chunk_pieces - 1) / chunk_pieces;
+  if (nch > kMaxChunks) return false;
   const int64_t slot_bytes = 2 * chunk_pieces * 16;
-  int64_t nslot = ring_bytes / slot_bytes;
-  if (nslot > kMaxSlots) nslot = kMaxSlots;
-  // Sweep 1 may run ahead of sweep 2 by as many rows as the ring holds (two, when sweep 2 has
-  // already released a row without a gradient); the exchange buffers and barriers are two deep,
-  // so the ring must not hold two whole rows.
-  if (nslot > 2 * nch - 1) nslot = 2 * nch - 1;
-  if (nslot < 1) return false;
-  if (has_grad && nslot < nch + (nch >= 2 ? 1 : 0)) return false;   // a row stays until sweep 2
-  if ((int64_t)cl * ns1 > kMaxRec1 && has_grad) return false;
-  if ((int64_t)cl * ns2 > kMaxRec2) return false;
-  if (!has_grad && cl * ns1 > kMaxRec1) return false;
+  const int64_t nslot = slots_bytes / slot_bytes;
+  if (nslot < 2) return false;
+  int64_t nres = 0, nring = 0;
+  if (!has_grad) {
+    nring = nslot < kMaxRing ? nslot : kMaxRing;   // nothing is read twice
+  } else {
+    // About 0.42 of the slice resident balances the HBM reads of the two sweeps (sweep 1 takes
+    // ~1.6x as long as sweep 2); the rest of the slots form the ring.
+    nres = (nch * 42 + 50) / 100;
+    if (nres > kMaxRes) nres = kMaxRes;
+    if (nres > nslot - 3) nres = nslot - 3;      // the ring keeps at least three slots in flight
+    if (nres < 0) nres = 0;
+    nring = nslot - nres;
+    if (nring > kMaxRing) nring = kMaxRing;
+    if (nres == nch) nring = 0;                    // everything resident: no stream
+  }
   plan.cl = cl;
-  plan.ns1 = ns1;
-  plan.ns2 = ns2;
   plan.nch = (int)nch;
-  plan.nslot = (int)nslot;
+  plan.nres = (int)nres;
+  plan.nring = (int)nring;
   plan.chunk_pieces = (int)chunk_pieces;
   plan.per_rank_pieces = (int)per_rank;
   plan.slot_bytes = (uint32_t)slot_bytes;
@@ -900,7 +893,7 @@ bool plan_for_cluster(int64_t pieces_total, int cl, bool has_grad, StagedPlan& p
 }
 
 int plan_smem_bytes(const StagedPlan& plan) {
-  return kCtrlBytes + plan.nslot * (int)plan.slot_bytes;
+  return kCtrlBytes + (plan.nres + plan.nring) * (int)plan.slot_bytes;
 }
 
 template <typename TIn, typename TOut>
@@ -923,9 +916,9 @@ cudaError_t max_clusters_for(const StagedPlan& plan, int sm_count, int& max_clus
   return cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg);
 }
 
-// The cluster size is chosen once per (device, shape class): among the sizes whose slice fits the
-// ring, the one that keeps the most SMs busy (cluster sizes that do not divide a GPC's SM count
-// leave SMs idle), then the smaller cluster.
+// The cluster size is chosen once per (device, shape class): the one that keeps the most SMs busy
+// (cluster sizes that do not divide a GPC's SM count leave SMs idle) among those whose streamed
+// bytes fit the L2 budget, else the one with the fewest streamed bytes.
 struct PlanKey {
   int dev, dtype, grad_dtype, has_grad;
   int64_t pieces_total;
@@ -952,7 +945,11 @@ bool choose_plan(int64_t pieces_total, bool has_grad, int sm_count, StagedPlan& 
       continue;
     }
     if (clusters < 1) continue;
-    const double score = (double)clusters * cl - 1e-3 * cl;
+    const double ctas = (double)clusters * cl;
+    const double streamed = ctas * (double)(plan.nch - plan.nres) * plan.slot_bytes;
+    double score = ctas;
+    if (has_grad && streamed > kL2BudgetBytes) score *= kL2BudgetBytes / streamed;
+    score -= 1e-3 * cl;
     if (score > best_score) {
       best_score = score;
       best = plan;
