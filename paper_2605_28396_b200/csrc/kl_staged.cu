@@ -66,10 +66,23 @@ struct StagedPlan {
   int nch;                // chunks per slice (same for every rank)
   int nres;               // resident chunks per slice
   int nring;              // stream-ring slots
+  int lead;               // leading streamed chunks of a slice that sweep 1 takes one row ahead
   int chunk_pieces;       // 16-byte pieces per chunk (per array)
   int per_rank_pieces;    // pieces per slice (last rank may own fewer)
   int num_clusters;
   uint32_t slot_bytes;    // 2 * chunk_pieces * 16
+};
+
+// What the consumers need to know about a row: which global row it is, whether its gradient is
+// written, its sampled token and the two logits at that token (at element 0 when the token is out
+// of range).  One lane loads these ahead of time so that the consumers hold no prefetch state.
+constexpr int kMetaDepth = 4;
+struct __align__(16) RowMeta {
+  int64_t r;
+  int y;
+  int wg;
+  float zy, uy;
+  int pad[2];
 };
 
 struct __align__(16) Ctrl {
@@ -84,6 +97,9 @@ struct __align__(16) Ctrl {
   float xbuf[2][kMaxRec][8];   // per row parity: one record per (rank, warp)
   float sbuf[kMaxRec][8];      // records of the running-maximum fallback
   int16_t tab[kMaxChunks];     // chunk j -> resident slot k (>= 0) or -1 (streamed)
+  RowMeta meta[kMetaDepth];    // row metadata, filled a few rows ahead by the metadata lane
+  unsigned long long meta_full[kMetaDepth];
+  unsigned long long meta_empty[kMetaDepth];
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
@@ -411,6 +427,10 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
     mbar_init(smem_u32(&ctrl.xbar[0]), cl * kNW);
     mbar_init(smem_u32(&ctrl.xbar[1]), cl * kNW);
     mbar_init(smem_u32(&ctrl.sbar), cl * kNW);
+    for (int s = 0; s < kMetaDepth; ++s) {
+      mbar_init(smem_u32(&ctrl.meta_full[s]), 1);
+      mbar_init(smem_u32(&ctrl.meta_empty[s]), kNW);
+    }
     ctrl.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -442,8 +462,6 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
 
   if (warp == kProducerWarp && lane == 0) {
     // ------------------------------------------------------------------ ring producer
-    // Order of the stream: per row, the streamed chunks for sweep 1, then (rows whose gradient is
-    // written) the same chunks again for sweep 2.
     if (nring > 0 && nres < nch) {
       int slot = 0;
       uint32_t phase = 0;
@@ -451,25 +469,34 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       RowCursor cur;
       cur.init(p);
       bool stop = false;
-      for (int64_t i = 0; i < my_rows && !stop && !*abort; ++i) {
-        bool wg;
-        const int64_t r = cur.locate(p, cluster_id + i * plan.num_clusters, wg);
-        for (int sweep = 0; sweep < (wg ? 2 : 1) && !stop; ++sweep) {
-          for (int j = 0; j < nch; ++j) {
-            if (ctrl.tab[j] >= 0) continue;
-            if (fills >= nring &&
-                !bounded_wait<false>(smem_u32(&ctrl.ring_empty[slot]), phase ^ 1u, abort)) {
-              stop = true;   // gave up: never overwrite a slot that may still be read
-              break;
-            }
-            issue_chunk(r, j, ring_base + (size_t)slot * plan.slot_bytes, &ctrl.ring_full[slot]);
-            ++fills;
-            if (++slot == nring) {
-              slot = 0;
-              phase ^= 1u;
-            }
+      // streamed chunks j in [j0, j1) of row r, in order
+      auto emit = [&](int64_t r, int j0, int j1) {
+        for (int j = j0; j < j1 && !stop; ++j) {
+          if (ctrl.tab[j] >= 0) continue;
+          if (fills >= nring &&
+              !bounded_wait<false>(smem_u32(&ctrl.ring_empty[slot]), phase ^ 1u, abort)) {
+            stop = true;   // gave up: never overwrite a slot that may still be read
+            return;
+          }
+          issue_chunk(r, j, ring_base + (size_t)slot * plan.slot_bytes, &ctrl.ring_full[slot]);
+          ++fills;
+          if (++slot == nring) {
+            slot = 0;
+            phase ^= 1u;
           }
         }
+      };
+      // Order of the stream (the consumers walk it in the same order): sweep 1 of row i from
+      // chunk `lead` on (row 0: from chunk 0), then the leading chunks of row i+1, then (rows
+      // whose gradient is written) all streamed chunks of row i again for sweep 2.
+      const int lead = plan.lead;
+      for (int64_t i = 0; i < my_rows && !stop && !*abort; ++i) {
+        bool wg, wg_next;
+        const int64_t r = cur.locate(p, cluster_id + i * plan.num_clusters, wg);
+        emit(r, i == 0 ? 0 : lead, nch);
+        if (i + 1 < my_rows)
+          emit(cur.locate(p, cluster_id + (i + 1) * plan.num_clusters, wg_next), 0, lead);
+        if (wg) emit(r, 0, nch);
       }
       // Drain: every copy this CTA issued must have landed before its shared memory goes away.
       int64_t pending = fills < nring ? fills : nring;
@@ -525,6 +552,29 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       }
       if (gave_up) atomicOr(p.status, ADWIN_DEV_TIMEOUT);
     }
+  } else if (warp == kProducerWarp && lane == 2) {
+    // ------------------------------------------------------------------ metadata lane
+    RowCursor cur;
+    cur.init(p);
+    for (int64_t i = 0; i < my_rows && !*abort; ++i) {
+      const int ms = (int)(i % kMetaDepth);
+      if (i >= kMetaDepth &&
+          !bounded_wait<false>(smem_u32(&ctrl.meta_empty[ms]),
+                               (uint32_t)((i / kMetaDepth - 1) & 1), abort))
+        break;
+      bool wg;
+      const int64_t r = cur.locate(p, cluster_id + i * plan.num_clusters, wg);
+      const int y = p.tokens[r];
+      float zy, uy;
+      fetch_logits_at<TIn>(p, r, y, zy, uy);
+      RowMeta& m = ctrl.meta[ms];
+      m.r = r;
+      m.y = y;
+      m.wg = wg ? 1 : 0;
+      m.zy = zy;
+      m.uy = uy;
+      mbar_arrive(smem_u32(&ctrl.meta_full[ms]));   // release: the fields are visible
+    }
   } else if (warp < kNW) {
     // ------------------------------------------------------------------ consumer warps
     const bool full_mode = (p.mode == ADWIN_GRAD_FULL_KL);
@@ -537,89 +587,120 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
     int64_t r_prev = 0;
     bool wg_prev = false;
 
-    // metadata pipeline: current row (C) and next row (N) held in registers
-    RowCursor cur;
-    cur.init(p);
-    int64_t rC = 0, rN = 0;
-    int yC = 0, yN = 0;
-    float zyC = 0.f, uyC = 0.f;
-    bool wgC = false, wgN = false;
-    cur.fetch_row(p, cluster_id, 0 < my_rows, rC, yC, wgC);
-    if (my_rows > 0) fetch_logits_at<TIn>(p, rC, yC, zyC, uyC);
-    cur.fetch_row(p, cluster_id + plan.num_clusters, 1 < my_rows, rN, yN, wgN);
-
     const int grp = warp / kGW;                  // this warp's group: chunks j % kG == grp
     const int gt = tid - grp * kGT;              // thread index inside the group
     const uint32_t toff = (uint32_t)gt * 16u;    // first of this thread's kP pieces in a chunk
     const int64_t iters = my_rows > 0 ? my_rows + 1 : 0;   // + one exchange for the last norm
+    Acc2 a;        // sweep-1 sums; carries the leading chunks of the next row across sweep 2
+    a.reset();
     for (int64_t i = 0; i < iters; ++i) {
       const bool real = i < my_rows;
-      // next rows' dependent loads, consumed one iteration later
-      float zyN = 0.f, uyN = 0.f;
-      int64_t rNN = 0;
-      int yNN = 0;
-      bool wgNN = false;
-      if (i + 1 < my_rows) fetch_logits_at<TIn>(p, rN, yN, zyN, uyN);
-      cur.fetch_row(p, cluster_id + (i + 2) * plan.num_clusters, i + 2 < my_rows, rNN, yNN, wgNN);
-
+      // this row's metadata (the flush iteration has none)
+      int64_t rC = 0;
+      int yC = 0;
+      float zyC = 0.f, uyC = 0.f;
+      bool wgC = false;
+      if (real) {
+        const int ms = (int)(i % kMetaDepth);
+        if (!bounded_wait<false>(smem_u32(&ctrl.meta_full[ms]),
+                                 (uint32_t)((i / kMetaDepth) & 1), abort)) {
+          timed_out = true;
+          break;
+        }
+        const RowMeta& m = ctrl.meta[ms];
+        rC = m.r;
+        yC = m.y;
+        wgC = m.wg != 0;
+        zyC = m.zy;
+        uyC = m.uy;
+      }
       const bool y_valid = (yC >= 0) && ((int64_t)yC < p.V);
       const float ref_s = zyC * kLog2e, ref_t = uyC * kLog2e;   // shared references of the row
       const float dref = wgC ? 0.f : zyC - uyC;                 // delta is centred on probe rows
       const uint32_t rpar = (uint32_t)(i & 1);                  // fill parity of resident slots
 
       // ---------------------------------------------------------------- sweep 1
-      Acc2 a;
-      a.reset();
-      if (real) {
-        const f2_t nrefs = splat2(-ref_s), nreft = splat2(-ref_t), ndref = splat2(-dref);
-        for (int j = 0; j < nch; ++j) {
-          const int k = ctrl.tab[j];
-          if (j % kG == grp) {
-            const char* sl;
-            if (k >= 0) {
-              if (!bounded_wait<false>(smem_u32(&ctrl.res_full[k]), rpar, abort)) timed_out = true;
-              sl = res_base + (size_t)k * plan.slot_bytes + toff;
-            } else {
-              if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort)) timed_out = true;
-              sl = ring_base + (size_t)rc_slot * plan.slot_bytes + toff;
+      // Visits v in [v0, nch) are chunks of row i (its leading chunks were taken one iteration
+      // earlier); at v == nch the row's record is posted to every CTA; visits v in (nch, vend)
+      // are the leading streamed chunks of row i+1, taken while the exchange is in flight.
+      const int par = (int)(i & 1);
+      {
+        const int v0 = real ? (i == 0 ? 0 : plan.lead) : nch;
+        const int vend = (real && i + 1 < my_rows) ? nch + plan.lead : nch;
+        bool wgv = wgC;
+        f2_t nrefs = splat2(-ref_s), nreft = splat2(-ref_t), ndref = splat2(-dref);
+        for (int v = v0;; ++v) {
+          if (v == nch) {
+            // record = { S, A, St, B0, B1, B2, q_prev, 0 }: this warp's sums over its lanes.
+            const float v0s = lane_sum(hsum2(a.S)), v1 = lane_sum(hsum2(a.A)), v2 = lane_sum(hsum2(a.St));
+            float v3 = 0.f, v4 = 0.f, v5 = 0.f;
+            if (real && !wgC) {
+              v3 = lane_sum(hsum2(a.B0));
+              v4 = lane_sum(hsum2(a.B1));
+              v5 = lane_sum(hsum2(a.B2));
             }
-            if (timed_out) break;
-            // The thread's pieces go to registers first and the slot is handed back at once, so
-            // the refill is in flight while the arithmetic runs.
-            const int np = pieces_in_chunk(j);
-            uint4 zr[kP], ur[kP];
-#pragma unroll
-            for (int h = 0; h < kP; ++h) {
-              if (gt + h * kGT < np) {
-                zr[h] = *reinterpret_cast<const uint4*>(sl + h * kGT * 16);
-                ur[h] = *reinterpret_cast<const uint4*>(sl + u_off + h * kGT * 16);
-              }
+            if (lane < cl) {
+              const uint32_t dst =
+                  map_to_rank(smem_u32(&ctrl.xbuf[par][rank * kNW + warp][0]), (uint32_t)lane);
+              remote_store4(dst, v0s, v1, v2, v3);
+              remote_store4(dst + 16, v4, v5, q_prev, 0.f);
+              remote_arrive_release(map_to_rank(smem_u32(&ctrl.xbar[par]), (uint32_t)lane));
             }
-            if (k < 0 || !wgC) {
-              __syncwarp();
-              if (lane == 0)
-                mbar_arrive(smem_u32(k < 0 ? &ctrl.ring_empty[rc_slot] : &ctrl.res_empty[k]));
-            }
-#pragma unroll
-            for (int h = 0; h < kP; ++h) {
-              if (gt + h * kGT < np) {
-                f2_t Z[NP], U[NP];
-                Pairs<TIn>::make(zr[h], Z);
-                Pairs<TIn>::make(ur[h], U);
-                if (wgC)
-                  acc_grad<NP>(Z, U, nrefs, nreft, a);
-                else
-                  acc_probe<NP>(Z, U, nrefs, nreft, ndref, a);
-              }
-            }
-          } else if (k < 0) {
-            // Not this group's chunk, but every warp observes and releases every fill of a ring
-            // slot: a parity wait is only sound within one phase of the barrier's current one.
-            if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort)) {
+            a.reset();
+            if (nch >= vend) break;
+            // from here on: row i+1
+            const int msn = (int)((i + 1) % kMetaDepth);
+            if (!bounded_wait<false>(smem_u32(&ctrl.meta_full[msn]),
+                                     (uint32_t)(((i + 1) / kMetaDepth) & 1), abort)) {
               timed_out = true;
               break;
             }
-            if (lane == 0) mbar_arrive(smem_u32(&ctrl.ring_empty[rc_slot]));
+            const RowMeta& mn = ctrl.meta[msn];
+            wgv = mn.wg != 0;
+            const float zyN = mn.zy, uyN = mn.uy;
+            nrefs = splat2(-zyN * kLog2e);
+            nreft = splat2(-uyN * kLog2e);
+            ndref = splat2(-(wgv ? 0.f : zyN - uyN));
+          }
+          if (v >= vend) break;   // (reached only when the leading chunks of row i+1 are done)
+          const int j = v < nch ? v : v - nch;
+          const int k = ctrl.tab[j];
+          const char* sl;
+          if (k >= 0) {   // resident chunks only occur in the part of row i (v < nch)
+            if (!bounded_wait<false>(smem_u32(&ctrl.res_full[k]), rpar, abort)) timed_out = true;
+            sl = res_base + (size_t)k * plan.slot_bytes + toff;
+          } else {
+            if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort)) timed_out = true;
+            sl = ring_base + (size_t)rc_slot * plan.slot_bytes + toff;
+          }
+          if (timed_out) break;
+          // The thread's pieces go to registers first and the slot is handed back at once, so
+          // the refill is in flight while the arithmetic runs.
+          const int np = pieces_in_chunk(j);
+          uint4 zr[kP], ur[kP];
+#pragma unroll
+          for (int h = 0; h < kP; ++h) {
+            if (gt + h * kGT < np) {
+              zr[h] = *reinterpret_cast<const uint4*>(sl + h * kGT * 16);
+              ur[h] = *reinterpret_cast<const uint4*>(sl + u_off + h * kGT * 16);
+            }
+          }
+          if (k < 0 || !wgv) {
+            __syncwarp();
+            if (lane == 0)
+              mbar_arrive(smem_u32(k < 0 ? &ctrl.ring_empty[rc_slot] : &ctrl.res_empty[k]));
+          }
+#pragma unroll
+          for (int h = 0; h < kP; ++h) {
+            if (gt + h * kGT < np) {
+              f2_t Z[NP], U[NP];
+              Pairs<TIn>::make(zr[h], Z);
+              Pairs<TIn>::make(ur[h], U);
+              if (wgv)
+                acc_grad<NP>(Z, U, nrefs, nreft, a);
+              else
+                acc_probe<NP>(Z, U, nrefs, nreft, ndref, a);
+            }
           }
           if (k < 0 && ++rc_slot == nring) {   // the ring cursor walks every streamed chunk
             rc_slot = 0;
@@ -630,25 +711,9 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       }
 
       // ---------------------------------------------------------------- exchange
-      // record = { S, A, St, B0, B1, B2, q_prev, 0 }: this warp's sums over its lanes.
       RowTotals t;
       float qtot;
       {
-        const float v0 = lane_sum(hsum2(a.S)), v1 = lane_sum(hsum2(a.A)), v2 = lane_sum(hsum2(a.St));
-        float v3 = 0.f, v4 = 0.f, v5 = 0.f;
-        if (real && !wgC) {
-          v3 = lane_sum(hsum2(a.B0));
-          v4 = lane_sum(hsum2(a.B1));
-          v5 = lane_sum(hsum2(a.B2));
-        }
-        const int par = (int)(i & 1);
-        if (lane < cl) {
-          const uint32_t dst =
-              map_to_rank(smem_u32(&ctrl.xbuf[par][rank * kNW + warp][0]), (uint32_t)lane);
-          remote_store4(dst, v0, v1, v2, v3);
-          remote_store4(dst + 16, v4, v5, q_prev, 0.f);
-          remote_arrive_release(map_to_rank(smem_u32(&ctrl.xbar[par]), (uint32_t)lane));
-        }
         if (!bounded_wait<true>(smem_u32(&ctrl.xbar[par]), (uint32_t)((i >> 1) & 1), abort)) {
           timed_out = true;
           break;
@@ -829,10 +894,9 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       }
       r_prev = rC;
       wg_prev = wgC;
-
-      // rotate the metadata pipeline
-      rC = rN; yC = yN; wgC = wgN; zyC = zyN; uyC = uyN;
-      rN = rNN; yN = yNN; wgN = wgNN;
+      // done with this row's metadata slot
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctrl.meta_empty[i % kMetaDepth]));
     }
     if (timed_out && lane == 0) {
       atomicOr(p.status, ADWIN_DEV_TIMEOUT);
@@ -886,6 +950,14 @@ bool plan_for_cluster(int64_t pieces_total, int cl, bool has_grad, StagedPlan& p
   plan.nch = (int)nch;
   plan.nres = (int)nres;
   plan.nring = (int)nring;
+  {
+    // Sweep 1 of the next row starts on its leading streamed chunks while the exchange of the
+    // current row is in flight (at most 3 chunks, and never the whole slice).
+    int lead = 0;
+    while (lead < 3 && lead + 1 < nch && ((lead + 1) * nres) / nch == (lead * nres) / nch) ++lead;
+    if (nring < 2) lead = 0;
+    plan.lead = lead;
+  }
   plan.chunk_pieces = (int)chunk_pieces;
   plan.per_rank_pieces = (int)per_rank;
   plan.slot_bytes = (uint32_t)slot_bytes;
