@@ -62,8 +62,8 @@ def measured_peak():
 
 # DRAM bytes per processed row of the staged kernel, from the committed ncu capture
 # (profiles/kl_staged_bf16_small_case_full.md), valid for the kernel source with this fingerprint.
-TRAFFIC_BYTES_PER_ROW = 872816
-TRAFFIC_KERNEL_SHA = "94f2eb9e27e29e8d"
+TRAFFIC_BYTES_PER_ROW = 1092165
+TRAFFIC_KERNEL_SHA = "bb178ae281615e9b"
 
 
 def recorded_traffic(rows):
@@ -215,6 +215,20 @@ def pinned_window_rows(batch, grad_dtype):
     return host
 
 
+def aggregate_over_ranks(times_ms, rows, device, world):
+    """Whole-job figures from per-rank ones: every time is the MAX over ranks (the job is as slow
+    as its slowest rank), the row count is the SUM (each rank processes its own batch, no
+    data-path collective).  Works on any backend (nccl on GPUs, gloo in the CPU test)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    r = torch.tensor([float(rows)], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(r, op=dist.ReduceOp.SUM)
+    return [float(x) for x in t], float(r[0])
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -287,13 +301,7 @@ def run_ours(args):
         raise SystemExit(f"device status {bits}: the timed run is invalid")
     loss = float(tot[0].item())
 
-    t = torch.tensor([ms_total, kernel_ms], dtype=torch.float64, device=dev)
-    r = torch.tensor([float(rows)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.all_reduce(r, op=dist.ReduceOp.SUM)
-    ms_total, kernel_ms = float(t[0]), float(t[1])
-    rows_all = float(r[0])
+    (ms_total, kernel_ms), rows_all = aggregate_over_ranks([ms_total, kernel_ms], rows, dev, world)
     ms_step = ms_total / args.steps
     value = rows_all / (ms_step / 1e3)
 
@@ -323,10 +331,7 @@ def run_ours(args):
         barrier()
         wall = (time.perf_counter() - h0) * 1e3
         ems = max(e0.elapsed_time(e1), wall) / args.e2e_steps
-        et = torch.tensor([ems], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(et, op=dist.ReduceOp.MAX)
-        ems = float(et[0])
+        (ems,), _ = aggregate_over_ranks([ems], rows, dev, world)
         h2d = rows * V * 2 * 2 + rows * 4
         d2h = rows * V * 2 + 3 * rows * 4
         same = bool(torch.allclose(hout.kl, out.kl.cpu(), rtol=1e-5, atol=1e-6))

@@ -301,3 +301,87 @@ def test_host_buffer_entry_point_matches_device_entry_point(flags):
     with pytest.raises(api.AdwinError):
         api.adwin_opd_kl_fwd_bwd_host(s_h, t_h, tok_h, torch.tensor([-1, 2, 3], dtype=torch.int32),
                                       None, device=DEV)
+
+
+def _oracle_on_rows(batch, rows, **kw):
+    """Oracle on selected (b, t) rows only: each row becomes a one-token sequence inside its window."""
+    bs = torch.tensor([b for b, _ in rows], device=batch.student.device)
+    ts = torch.tensor([t for _, t in rows], device=batch.student.device)
+    s = synth.bits_for_oracle(batch.student[bs, ts].unsqueeze(1))
+    t = synth.bits_for_oracle(batch.teacher[bs, ts].unsqueeze(1))
+    tok = batch.tokens[bs, ts].unsqueeze(1).cpu().numpy()
+    return O.opd_kl_fwd_bwd(s, t, tok, np.ones(len(rows), np.int32), None, **kw)
+
+
+def _sample_rows(limits, per_seq, rng):
+    """First, last and a few random processed rows of every sequence."""
+    rows = []
+    for b, n in enumerate(limits):
+        if n <= 0:
+            continue
+        ts = {0, int(n) - 1} | {int(x) for x in rng.integers(0, int(n), size=per_seq)}
+        rows += [(b, t) for t in sorted(ts)]
+    return rows
+
+
+def test_config3_full_size_in_the_bench_launch_configuration_on_sampled_rows():
+    """The workload bench.py times, at full size, with the oracle on sampled rows plus the
+    properties that hold at any size (untouched tail, zeroed scalars, reproducible sums)."""
+    batch = synth.make_batch(3, device=DEV)
+    B, T, V = batch.shape
+    sentinel = 7.0
+    grad = torch.full((B, T, V), sentinel, dtype=torch.bfloat16, device=DEV)
+    got = api.adwin_opd_kl_fwd_bwd(batch.student, batch.teacher, batch.tokens, batch.window,
+                                   batch.rollout_len, grad=grad)
+    torch.cuda.synchronize()
+    api.raise_on_dev_status(got.dev_status)
+    w = batch.window.cpu().numpy()
+    rows = _sample_rows(w, 2, np.random.default_rng(3))
+    ref = _oracle_on_rows(batch, rows)
+    bs = torch.tensor([b for b, _ in rows], device=DEV)
+    ts = torch.tensor([t for _, t in rows], device=DEV)
+    sub = type("S", (), {})()
+    sub.kl, sub.logratio, sub.gsq = (x[bs, ts].unsqueeze(1) for x in (got.kl, got.logratio, got.gsq))
+    ones = np.ones((len(rows), 1), dtype=bool)
+    P.check_scalars(sub, ref, 2e-3, ones, grad_mask=ones)
+    P.check_grad_rows(grad[bs, ts].double().cpu().numpy(), ref["grad"][:, 0], 2e-3, store=2.0 ** -8)
+    for b in range(B):                                   # rows past the window: never touched
+        assert (grad[b, int(w[b]):] == sentinel).all()
+        assert (got.kl[b, int(w[b]):] == 0).all() and (got.gsq[b, int(w[b]):] == 0).all()
+    seq, tot = api.adwin_window_reduce(got.kl, got.logratio, got.gsq, batch.window, batch.rollout_len)
+    torch.cuda.synchronize()
+    mask = torch.arange(T, device=DEV)[None, :] < batch.window[:, None]
+    want = (got.kl.double() * mask).sum()
+    assert abs(tot[0].item() - want.item()) <= 1e-9 * abs(want.item())
+    assert tot[3].item() == float(w.sum()) and torch.isfinite(got.kl).all() and (got.kl[mask] > -1e-4).all()
+
+
+def test_config4_full_size_probe_pass_on_sampled_rows():
+    """Delayed full-rollout probe at full size (B=8, T=8192, V=151936, ragged rollouts): one pass
+    without a gradient, then the alignment audit; oracle on sampled rows, audit against the oracle's
+    audit of the same per-token scalars."""
+    batch = synth.make_batch(4, device=DEV, ragged_rollout=True, fill_all_rows=False)
+    B, T, V = batch.shape
+    got = api.adwin_opd_kl_fwd_bwd(batch.student, batch.teacher, batch.tokens, batch.window,
+                                   batch.rollout_len, flags=api.RANGE_FULL)
+    torch.cuda.synchronize()
+    api.raise_on_dev_status(got.dev_status)
+    w, r = batch.window.cpu().numpy(), batch.rollout_len.cpu().numpy()
+    rows = _sample_rows(r, 3, np.random.default_rng(4))
+    ref = _oracle_on_rows(batch, rows, want_grad=False)
+    bs = torch.tensor([b for b, _ in rows], device=DEV)
+    ts = torch.tensor([t for _, t in rows], device=DEV)
+    sub = type("S", (), {})()
+    sub.kl, sub.logratio, sub.gsq = (x[bs, ts].unsqueeze(1) for x in (got.kl, got.logratio, got.gsq))
+    P.check_scalars(sub, ref, 2e-3, np.ones((len(rows), 1), dtype=bool))
+    for b in range(B):
+        assert (got.kl[b, int(r[b]):] == 0).all()
+    al = api.adwin_probe_align(got.kl, got.logratio, got.gsq, batch.window, batch.rollout_len)
+    torch.cuda.synchronize()
+    same = O.probe_align(got.kl.cpu().numpy(), got.logratio.cpu().numpy(), got.gsq.cpu().numpy(),
+                         w, r, np.array(api.DEFAULT_CANDIDATES, np.int32), api.RHO_STAR)
+    np.testing.assert_allclose(al.batch_stats.cpu().numpy(), same["batch_stats"], rtol=1e-12)
+    np.testing.assert_allclose(al.seq_stats.cpu().numpy(), same["seq_stats"], rtol=1e-12, atol=1e-12)
+    assert int(al.L_next.item()) == same["L_next"] and int(al.flags.item()) == same["flags"]
+    rho = al.batch_stats[:, 0].cpu().numpy()
+    assert (np.diff(rho[:-1]) >= -1e-12).all() and (rho <= 1 + 1e-12).all()
