@@ -43,6 +43,7 @@
 
 namespace adwin {
 
+constexpr int kLeadMax = 2;          // chunks of the next row that sweep 1 takes during the exchange
 constexpr int kNT = 480;             // consumer threads (512 in all: the block keeps 128 registers per thread)
 constexpr int kNW = kNT / 32;        // consumer warps
 constexpr int kG = 1;                // consumer groups: group g takes the chunks j with j % kG == g
@@ -162,6 +163,26 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
           "r"(dst),
       "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+// L2 eviction priorities for the bulk copies: a chunk that will be fetched again by sweep 2 should
+// outlive the chunks that are read only once.
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_load_hint(uint32_t dst, const void* src, uint32_t bytes,
+                                               uint32_t bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1], %2, [%3], %4;" ::"r"(dst),
+      "l"(src), "r"(bytes), "r"(bar), "l"(pol)
       : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
@@ -443,7 +464,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
     return left < plan.chunk_pieces ? left : plan.chunk_pieces;
   };
   // issue the two bulk copies of chunk j of row r into a slot
-  auto issue_chunk = [&](int64_t r, int j, char* slot, unsigned long long* full) {
+  auto issue_chunk = [&](int64_t r, int j, char* slot, unsigned long long* full, uint64_t pol) {
     int np = pieces_in_chunk(j);
     np = np < 0 ? 0 : np;
     const uint32_t bytes = (uint32_t)np * 16u;
@@ -455,8 +476,8 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
                           (size_t)j * plan.chunk_pieces * 16;
       mbar_arrive_expect_tx(bar, 2u * bytes);
       const uint32_t dst = smem_u32(slot);
-      bulk_load(dst, static_cast<const char*>(p.student) + goff, bytes, bar);
-      bulk_load(dst + u_off, static_cast<const char*>(p.teacher) + goff, bytes, bar);
+      bulk_load_hint(dst, static_cast<const char*>(p.student) + goff, bytes, bar, pol);
+      bulk_load_hint(dst + u_off, static_cast<const char*>(p.teacher) + goff, bytes, bar, pol);
     }
   };
 
@@ -470,7 +491,9 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       cur.init(p);
       bool stop = false;
       // streamed chunks j in [j0, j1) of row r, in order
-      auto emit = [&](int64_t r, int j0, int j1) {
+      const uint64_t pol_keep = l2_policy_evict_last();
+      const uint64_t pol_once = l2_policy_evict_first();
+      auto emit = [&](int64_t r, int j0, int j1, uint64_t pol) {
         for (int j = j0; j < j1 && !stop; ++j) {
           if (ctrl.tab[j] >= 0) continue;
           if (fills >= nring &&
@@ -478,7 +501,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
             stop = true;   // gave up: never overwrite a slot that may still be read
             return;
           }
-          issue_chunk(r, j, ring_base + (size_t)slot * plan.slot_bytes, &ctrl.ring_full[slot]);
+          issue_chunk(r, j, ring_base + (size_t)slot * plan.slot_bytes, &ctrl.ring_full[slot], pol);
           ++fills;
           if (++slot == nring) {
             slot = 0;
@@ -493,10 +516,13 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       for (int64_t i = 0; i < my_rows && !stop && !*abort; ++i) {
         bool wg, wg_next;
         const int64_t r = cur.locate(p, cluster_id + i * plan.num_clusters, wg);
-        emit(r, i == 0 ? 0 : lead, nch);
-        if (i + 1 < my_rows)
-          emit(cur.locate(p, cluster_id + (i + 1) * plan.num_clusters, wg_next), 0, lead);
-        if (wg) emit(r, 0, nch);
+        // first fetch of a chunk that sweep 2 fetches again: keep it in L2; last fetch: let it go
+        emit(r, i == 0 ? 0 : lead, nch, wg ? pol_keep : pol_once);
+        if (i + 1 < my_rows) {
+          const int64_t rn = cur.locate(p, cluster_id + (i + 1) * plan.num_clusters, wg_next);
+          emit(rn, 0, lead, wg_next ? pol_keep : pol_once);
+        }
+        if (wg) emit(r, 0, nch, pol_once);
       }
       // Drain: every copy this CTA issued must have landed before its shared memory goes away.
       int64_t pending = fills < nring ? fills : nring;
@@ -522,6 +548,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
     if (nres > 0) {
       RowCursor cur;
       cur.init(p);
+      const uint64_t pol_once = l2_policy_evict_first();   // resident chunks are fetched once
       int64_t last_row = -1;   // last row some slot was filled for, and how many slots got it
       int last_k = 0;
       for (int64_t i = 0; i < my_rows && !*abort; ++i) {
@@ -533,7 +560,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
           if (i > 0 &&
               !bounded_wait<false>(smem_u32(&ctrl.res_empty[k]), (uint32_t)((i - 1) & 1), abort))
             break;   // gave up: never overwrite a slot that may still be read
-          issue_chunk(r, j, res_base + (size_t)k * plan.slot_bytes, &ctrl.res_full[k]);
+          issue_chunk(r, j, res_base + (size_t)k * plan.slot_bytes, &ctrl.res_full[k], pol_once);
           last_row = i;
           last_k = k + 1;
         }
@@ -952,9 +979,9 @@ bool plan_for_cluster(int64_t pieces_total, int cl, bool has_grad, StagedPlan& p
   plan.nring = (int)nring;
   {
     // Sweep 1 of the next row starts on its leading streamed chunks while the exchange of the
-    // current row is in flight (at most 3 chunks, and never the whole slice).
+    // current row is in flight (at most kLeadMax chunks, and never the whole slice).
     int lead = 0;
-    while (lead < 3 && lead + 1 < nch && ((lead + 1) * nres) / nch == (lead * nres) / nch) ++lead;
+    while (lead < kLeadMax && lead + 1 < nch && ((lead + 1) * nres) / nch == (lead * nres) / nch) ++lead;
     if (nring < 2) lead = 0;
     plan.lead = lead;
   }
