@@ -967,7 +967,7 @@ bool plan_for_cluster(int64_t pieces_total, int cl, bool has_grad, StagedPlan& p
     // ~1.6x as long as sweep 2); the rest of the slots form the ring.
     nres = (nch * 42 + 50) / 100;
     if (nres > kMaxRes) nres = kMaxRes;
-    if (nres > nslot - 3) nres = nslot - 3;      // the ring keeps at least three slots in flight
+    if (nres > nslot - 2) nres = nslot - 2;      // the ring keeps at least two slots in flight
     if (nres < 0) nres = 0;
     nring = nslot - nres;
     if (nring > kMaxRing) nring = kMaxRing;
