@@ -844,6 +844,9 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       if (wgC) {
         const f2_t L2 = splat2(kLog2e), NEG1 = splat2(-1.f);
         const f2_t nM2s = splat2(-t.M2s), nc0 = splat2(-rs.c0), coef2 = splat2(rs.coef);
+        // bf16 logits: g = e * (coef*delta - coef*c0) saves one operation per pair; its rounding
+        // (relative to coef*delta, not to the difference) is far inside that dtype's tolerance.
+        const f2_t ncc0 = splat2(-rs.coef * rs.c0);
         const int64_t ypiece = y_valid ? ((int64_t)yC / N - piece0) : -1;   // slice-relative
         char* gthread = static_cast<char*>(p.grad) +
                         ((size_t)rC * p.ld_grad + (size_t)(piece0 + gt) * N) * sizeof(TOut);
@@ -882,8 +885,12 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
                 for (int e = 0; e < NP; ++e) {
                   const f2_t E = ex2_2(fma2(Z[e], L2, nM2s));
                   if (full_mode) {
-                    const f2_t D = add2(fma2(U[e], NEG1, Z[e]), nc0);
-                    G[e] = mul2(E, mul2(D, coef2));
+                    if (sizeof(TIn) == 2) {
+                      G[e] = mul2(E, fma2(fma2(U[e], NEG1, Z[e]), coef2, ncc0));
+                    } else {
+                      const f2_t D = add2(fma2(U[e], NEG1, Z[e]), nc0);
+                      G[e] = mul2(E, mul2(D, coef2));
+                    }
                   } else {
                     G[e] = mul2(E, coef2);
                   }
