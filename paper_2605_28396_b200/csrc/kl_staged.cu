@@ -285,12 +285,43 @@ __device__ __forceinline__ f2_t ex2_2(f2_t x) {
   upk2(x, a, b);
   return pk2(ex2f(a), ex2f(b));
 }
+__device__ __forceinline__ f2_t splat2(float v) { return pk2(v, v); }
+__device__ __forceinline__ f2_t sub2(f2_t a, f2_t b) {
+  f2_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// 2^x of a pair on the FMA pipe, to relieve the MUFU unit that bounds sweep 1.  x is clamped to
+// [-120, 105] (below that the term is nil against a sum >= 1; at the upper end the result exceeds
+// the limit that sends the row to the safe path), rounded to the nearest integer n by adding
+// 1.5*2^23, 2^(x-n) comes from a degree-4 polynomial on [-1/2, 1/2] (relative error < 2.7e-6,
+// mean 4e-8) and n is added to the exponent field.  A NaN comes out as a finite number: callers
+// keep a second, unclamped use of the input so that it still poisons the row.
+__device__ __forceinline__ f2_t ex2_poly2(f2_t x) {
+  float a, b;
+  upk2(x, a, b);
+  a = fminf(fmaxf(a, -120.f), 105.f);
+  b = fminf(fmaxf(b, -120.f), 105.f);
+  const f2_t xc = pk2(a, b);
+  const f2_t MG = splat2(12582912.f);
+  const f2_t t = add2(xc, MG);
+  const f2_t f = sub2(xc, sub2(t, MG));
+  f2_t q = fma2(splat2(9.570101276e-03f), f, splat2(5.591785908e-02f));
+  q = fma2(q, f, splat2(2.402474433e-01f));
+  q = fma2(q, f, splat2(6.931217909e-01f));
+  q = fma2(q, f, splat2(9.999992847e-01f));
+  float tl, th, ql, qh;
+  upk2(t, tl, th);
+  upk2(q, ql, qh);
+  const uint32_t rl = __float_as_uint(ql) + (__float_as_uint(tl) << 23);
+  const uint32_t rh = __float_as_uint(qh) + (__float_as_uint(th) << 23);
+  return pk2(__uint_as_float(rl), __uint_as_float(rh));
+}
 __device__ __forceinline__ float hsum2(f2_t v) {
   float a, b;
   upk2(v, a, b);
   return a + b;
 }
-__device__ __forceinline__ f2_t splat2(float v) { return pk2(v, v); }
 
 // A 16-byte piece as NP pairs of consecutive vocabulary entries.
 template <typename T>
@@ -322,8 +353,16 @@ struct Acc2 {
   }
 };
 
+// Teacher pairs per 16-byte piece whose exponential is evaluated on the FMA pipe: one of the four
+// pairs of a bf16 piece (more than that and the FMA/ALU pipes become the limit, measured); none
+// for fp32 logits, whose sweep has half the exponentials per byte and a 1e-5 tolerance.
+template <typename T>
+__host__ __device__ constexpr int kPolyPairs() { return sizeof(T) == 2 ? 1 : 0; }
+
 // Sweep 1, rows whose gradient is written: e = 2^(z log2e - ref_s), delta = z - u uncentred.
-template <int NP>
+// The first PT teacher pairs of a piece take their exponential from the polynomial (the teacher
+// sum only enters through its logarithm, and delta still sees the unclamped logits).
+template <int NP, int PT>
 __device__ __forceinline__ void acc_grad(const f2_t (&Z)[NP], const f2_t (&U)[NP], f2_t nrefs,
                                          f2_t nreft, Acc2& a) {
   const f2_t L2 = splat2(kLog2e), NEG1 = splat2(-1.f);
@@ -333,7 +372,8 @@ __device__ __forceinline__ void acc_grad(const f2_t (&Z)[NP], const f2_t (&U)[NP
     const f2_t D = fma2(U[i], NEG1, Z[i]);
     a.S = add2(a.S, E);
     a.A = fma2(E, D, a.A);
-    a.St = add2(a.St, ex2_2(fma2(U[i], L2, nreft)));
+    const f2_t xt = fma2(U[i], L2, nreft);
+    a.St = add2(a.St, (i < PT) ? ex2_poly2(xt) : ex2_2(xt));
   }
 }
 
@@ -724,7 +764,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
               Pairs<TIn>::make(zr[h], Z);
               Pairs<TIn>::make(ur[h], U);
               if (wgv)
-                acc_grad<NP>(Z, U, nrefs, nreft, a);
+                acc_grad<NP, kPolyPairs<TIn>()>(Z, U, nrefs, nreft, a);
               else
                 acc_probe<NP>(Z, U, nrefs, nreft, ndref, a);
             }

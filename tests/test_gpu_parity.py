@@ -129,6 +129,26 @@ def test_sampled_token_far_below_the_row_maximum(path, in_dt, g_dt):
     run_and_check(batch, grad_dtype=g_dt, grad_mode=api.GRAD_SAMPLED, flags=flags)
 
 
+@pytest.mark.parametrize("g_dt", [torch.bfloat16, None])
+def test_teacher_logits_outside_the_range_of_the_polynomial_exponential(g_dt):
+    """The staged kernel takes the exponential of the first teacher pair of every 16-byte piece
+    from a polynomial that is only valid on a clamped range: entries far below the reference must
+    still count as nil, and one far above it must still send the row to the safe path."""
+    batch = synth.make_batch(2, device=DEV, B=2, T=5, V=8192)
+    batch.window = torch.tensor([5, 3], dtype=torch.int32, device=DEV)
+    first_pair = torch.arange(0, 8192, 8, device=DEV)
+    batch.teacher[0, 1, first_pair[5:400]] = -3.0e4            # far below: 2^x underflows
+    batch.teacher[0, 1, first_pair[5:400] + 1] = -250.0
+    batch.teacher[1, 0, first_pair[::7]] = -1.0e3
+    uy = float(batch.teacher[0, 3, int(batch.tokens[0, 3])])
+    batch.teacher[0, 3, first_pair[17]] = uy + 96.0              # far above, polynomial position
+    uy = float(batch.teacher[1, 2, int(batch.tokens[1, 2])])
+    batch.teacher[1, 2, first_pair[900] + 1] = uy + 71.0         # just inside the clamp
+    flags = api.RANGE_FULL if g_dt is None else 0
+    run_and_check(batch, grad_dtype=g_dt, flags=flags)
+    run_and_check(batch, grad_dtype=g_dt, grad_mode=api.GRAD_SAMPLED, flags=flags)
+
+
 @pytest.mark.parametrize("V", [1, 2, 7, 8, 9, 1001, 4100, 65537])
 def test_odd_vocab_sizes(V):
     batch = synth.make_batch(2, device=DEV, B=2, T=6, V=V)
