@@ -342,6 +342,54 @@ double adwin_oracle_literal_cosine(const double *grad, const int32_t *rollout_le
   return (np_all > 0) ? dot_all / (sqrt(np_all) * sqrt(nf_all)) : 0.0;
 }
 
+/*
+ * Discounted return-to-go of the per-token costs (Eq. 3; G_t^gamma in the appendix that derives the
+ * OPD gradient), written out as the definition: for every position t inside the range,
+ *   G[b,t] = sum over t' from t to the last position of the range of gamma^(t'-t) * c[b,t'],
+ * one power and one product per term, no recurrence.  The range is the prefix window (t < W_b,
+ * t < R_b, t < T) or, with ORACLE_FLAG_RANGE_FULL, the rollout (t < R_b, t < T); positions outside
+ * it get 0.  gamma^0 = 1 also for gamma = 0 (C's pow), which gives G = c, the token-local case.
+ */
+void adwin_oracle_return_to_go(const double *c, const int32_t *window, const int32_t *rollout_len,
+                               int64_t B, int64_t T, double gamma, int flags, double *G) {
+  for (int64_t b = 0; b < B; ++b) {
+    int64_t W = window[b];
+    int64_t R = rollout_len ? rollout_len[b] : T;
+    for (int64_t t = 0; t < T; ++t) {
+      int in_t = (flags & ORACLE_FLAG_RANGE_FULL) ? (t < R && t < T) : (t < W && t < R && t < T);
+      double acc = 0.0, comp = 0.0;
+      if (in_t) {
+        for (int64_t tp = t; tp < T; ++tp) {
+          int in_tp = (flags & ORACLE_FLAG_RANGE_FULL) ? (tp < R) : (tp < W && tp < R);
+          if (!in_tp) break;
+          comp_add(&acc, &comp, pow(gamma, (double)(tp - t)) * c[b * T + tp]);
+        }
+      }
+      G[b * T + t] = acc + comp;
+    }
+  }
+}
+
+/*
+ * One position of the future-coupled estimator in logit space (Eq. 3): the sampled-token gradient
+ * of Eq. 4 with a given coefficient w in place of c_t,
+ *   g_k = alpha * w * (1[k = y] - p_k),    p = softmax(z),    gsq = sum_k g_k^2.
+ * y outside [0,V) gives a NaN gradient, like the SAMPLED mode of adwin_oracle_row.
+ */
+void adwin_oracle_row_weighted(const double *z, int64_t V, int64_t y, double alpha, double w,
+                               double *gsq, double *g) {
+  double ls = adwin_oracle_logsumexp(z, V);
+  double coef = (y >= 0 && y < V) ? alpha * w : NAN;
+  double q2 = 0.0, q2c = 0.0;
+  for (int64_t k = 0; k < V; ++k) {
+    double p = exp(z[k] - ls);
+    double gk = coef * ((k == y ? 1.0 : 0.0) - p);
+    if (g) g[k] = gk;
+    comp_add(&q2, &q2c, gk * gk);
+  }
+  *gsq = q2 + q2c;
+}
+
 int adwin_oracle_num_threads(void) {
 #ifdef _OPENMP
   extern int omp_get_max_threads(void);

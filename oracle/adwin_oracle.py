@@ -171,3 +171,26 @@ def literal_cosine(grad, rollout_len, L: int):
                                               ctypes.c_int64(T), ctypes.c_int64(V),
                                               ctypes.c_int64(int(L)), _p(per_seq))
     return float(micro), per_seq
+
+
+def return_to_go(logratio, window, rollout_len=None, gamma: float = 0.0, flags: int = 0):
+    """Discounted return-to-go G[b,t] of the per-token costs over each sequence's range (Eq. 3)."""
+    c = _f64(logratio)
+    B, T = c.shape
+    window, rollout_len = _i32(window), _i32(rollout_len)
+    G = np.empty((B, T), dtype=np.float64)
+    lib().adwin_oracle_return_to_go(_p(c), _p(window), _p(rollout_len), ctypes.c_int64(B),
+                                    ctypes.c_int64(T), ctypes.c_double(gamma), ctypes.c_int(flags),
+                                    _p(G))
+    return G
+
+
+def row_weighted(z, y: int, alpha: float, w: float):
+    """Sampled-token gradient of one position with coefficient w in place of c: (g, gsq)."""
+    z = _f64(z)
+    g = np.empty(z.size, dtype=np.float64)
+    gsq = ctypes.c_double()
+    lib().adwin_oracle_row_weighted(_p(z), ctypes.c_int64(z.size), ctypes.c_int64(int(y)),
+                                    ctypes.c_double(alpha), ctypes.c_double(w), ctypes.byref(gsq),
+                                    _p(g))
+    return g, gsq.value
