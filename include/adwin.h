@@ -159,6 +159,41 @@ int adwin_probe_align(const float* kl, const float* logratio, const float* gsq,
                       void* cuda_stream);
 
 /*
+ * Discounted return-to-go of the per-token costs (Eq. 3; the derivation of the OPD gradient in the
+ * appendix defines G_t^gamma):
+ *     rtg[b,t] = sum_{t' = t}^{E_b - 1} gamma^(t'-t) * logratio[b,t']      for t < E_b,   0 elsewhere,
+ * where E_b = min(W_b, R_b, T) is the end of the prefix window, or min(R_b, T) with
+ * ADWIN_RANGE_FULL (the only flag accepted).  gamma = 0 returns the costs themselves (the
+ * token-local estimator the paper trains with), gamma = 1 their suffix sums.
+ * logratio, rtg : [B,T] float32 DEVICE pointers (rtg may not alias logratio); window, rollout_len
+ * as in adwin_opd_kl_fwd_bwd (rollout_len may be NULL); out-of-range lengths are clamped to
+ * [0,T] here (adwin_opd_kl_fwd_bwd reports them).  gamma outside [0,1] (or NaN) returns
+ * ADWIN_ERR_SHAPE.  Sums are float64 in a fixed order; nothing is allocated or synchronised.
+ */
+int adwin_return_to_go(const float* logratio, const int32_t* window, const int32_t* rollout_len,
+                       int64_t B, int64_t T, double gamma, int flags, float* rtg,
+                       void* cuda_stream);
+
+/*
+ * adwin_opd_kl_fwd_bwd in ADWIN_GRAD_SAMPLED mode with a caller-supplied coefficient per
+ * position in place of c_t:   g_k = grad_scale * row_coef[b,t] * (1[k = y] - p_k),
+ * i.e. one term G_t * grad log pi_theta(y_t) of the future-coupled estimator (Eq. 3) in logit
+ * space.  With gamma > 0 the coefficient of position t depends on later positions, so the caller
+ * runs a read-only pass first (grad_student = NULL) for logratio, then adwin_return_to_go, then
+ * this call.  row_coef : [B,T] float32 DEVICE pointer, read at the processed positions only.
+ * All other arguments, outputs (kl, logratio, lse are those of the row; gsq is the squared norm
+ * of the weighted gradient), layouts and errors are those of adwin_opd_kl_fwd_bwd.
+ */
+int adwin_opd_kl_fwd_bwd_weighted(const void* student_logits, const void* teacher_logits,
+                                  int dtype, int64_t B, int64_t T, int64_t V, int64_t ld,
+                                  const int32_t* tokens, const int32_t* window,
+                                  const int32_t* rollout_len, const float* row_coef,
+                                  float grad_scale, int flags, void* grad_student, int grad_dtype,
+                                  int64_t ld_grad, float* kl, float* logratio, float* gsq,
+                                  float* lse_student, float* lse_teacher, void* workspace,
+                                  size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
+
+/*
  * The same pass for logits that live in HOST memory (pinned memory gives asynchronous copies).
  * Only the rows inside the processed range cross PCIe -- the window skip of Section 4.1 saves the
  * transfer as well as the arithmetic -- in stages of at most rows_per_stage rows of one sequence;

@@ -27,7 +27,8 @@ RHO_STAR = math.sqrt(2.0) / 2.0                          # Section 4.2, threshol
 EXPORTS = ("adwin_version", "adwin_status_string", "adwin_workspace_bytes",
            "adwin_opd_kl_fwd_bwd", "adwin_window_reduce", "adwin_probe_align",
            "adwin_host_staging_bytes", "adwin_opd_kl_fwd_bwd_host",
-           "adwin_no_alloc_max_sequences", "adwin_opd_kl_fwd_bwd_no_alloc")
+           "adwin_no_alloc_max_sequences", "adwin_opd_kl_fwd_bwd_no_alloc",
+           "adwin_return_to_go", "adwin_opd_kl_fwd_bwd_weighted")
 
 _lib = None
 
@@ -74,6 +75,13 @@ def lib():
         L.adwin_opd_kl_fwd_bwd_no_alloc.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, i64, vp,
                                                     vp, vp, f32, ctypes.c_int, ctypes.c_int, vp,
                                                     ctypes.c_int, i64, vp, vp, vp, vp, vp, vp, vp]
+        L.adwin_return_to_go.restype = ctypes.c_int
+        L.adwin_return_to_go.argtypes = [vp, vp, vp, i64, i64, f64, ctypes.c_int, vp, vp]
+        L.adwin_opd_kl_fwd_bwd_weighted.restype = ctypes.c_int
+        L.adwin_opd_kl_fwd_bwd_weighted.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, i64, vp,
+                                                    vp, vp, vp, f32, ctypes.c_int, vp,
+                                                    ctypes.c_int, i64, vp, vp, vp, vp, vp, vp, sz,
+                                                    vp, vp]
         _lib = L
     return _lib
 
@@ -105,7 +113,8 @@ def adwin_workspace_bytes(B, T, V, dtype=BF16, flags=0) -> int:
 
 def adwin_opd_kl_fwd_bwd(student, teacher, tokens, window, rollout_len=None, *, grad_scale=1.0,
                          grad_mode=GRAD_FULL_KL, flags=0, grad=None, grad_dtype=None,
-                         want_gsq=True, want_lse=False, out=None, workspace=None, dev_status=None):
+                         want_gsq=True, want_lse=False, out=None, workspace=None, dev_status=None,
+                         row_coef=None):
     """Windowed per-token OPD divergence, forward + backward (see include/adwin.h).
 
     student, teacher: [B,T,V] CUDA tensors (fp32 or bf16), last dim contiguous, rows at a uniform
@@ -113,6 +122,7 @@ def adwin_opd_kl_fwd_bwd(student, teacher, tokens, window, rollout_len=None, *, 
     allocated (uninitialised outside the window unless ZERO_TAIL), or both None for no gradient.
     Returns a namespace with kl, logratio, gsq, lse_s, lse_t, grad, dev_status (device tensors).
     Nothing is synchronised; read ``dev_status`` (or call ``raise_on_dev_status``) after a sync.
+    With ``row_coef`` (see ``adwin_opd_kl_fwd_bwd_weighted``) the call goes to that entry point.
     """
     assert student.is_cuda and teacher.is_cuda and student.shape == teacher.shape
     assert student.dim() == 3 and student.dtype == teacher.dtype
@@ -146,14 +156,43 @@ def adwin_opd_kl_fwd_bwd(student, teacher, tokens, window, rollout_len=None, *, 
         dev_status = torch.zeros(1, dtype=torch.int32, device=dev)
     o.dev_status = dev_status
     o.workspace = workspace
-    rc = lib().adwin_opd_kl_fwd_bwd(
-        _ptr(student), _ptr(teacher), _dtype_code(student.dtype), B, T, V, ld, _ptr(tokens),
-        _ptr(window), _ptr(rollout_len), float(grad_scale), int(grad_mode), int(flags), _ptr(grad),
-        _dtype_code(grad.dtype) if grad is not None else 0, ld_grad, _ptr(o.kl), _ptr(o.logratio),
-        _ptr(o.gsq), _ptr(o.lse_s), _ptr(o.lse_t), _ptr(workspace), workspace.numel(),
-        _ptr(dev_status), _stream(dev))
+    gdt = _dtype_code(grad.dtype) if grad is not None else 0
+    if row_coef is None:
+        rc = lib().adwin_opd_kl_fwd_bwd(
+            _ptr(student), _ptr(teacher), _dtype_code(student.dtype), B, T, V, ld, _ptr(tokens),
+            _ptr(window), _ptr(rollout_len), float(grad_scale), int(grad_mode), int(flags),
+            _ptr(grad), gdt, ld_grad, _ptr(o.kl), _ptr(o.logratio), _ptr(o.gsq), _ptr(o.lse_s),
+            _ptr(o.lse_t), _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream(dev))
+    else:
+        assert row_coef.shape == (B, T) and row_coef.dtype == torch.float32
+        assert row_coef.is_contiguous() and row_coef.device == dev
+        rc = lib().adwin_opd_kl_fwd_bwd_weighted(
+            _ptr(student), _ptr(teacher), _dtype_code(student.dtype), B, T, V, ld, _ptr(tokens),
+            _ptr(window), _ptr(rollout_len), _ptr(row_coef), float(grad_scale), int(flags),
+            _ptr(grad), gdt, ld_grad, _ptr(o.kl), _ptr(o.logratio), _ptr(o.gsq), _ptr(o.lse_s),
+            _ptr(o.lse_t), _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream(dev))
     _check(rc)
     return o
+
+
+def adwin_opd_kl_fwd_bwd_weighted(student, teacher, tokens, window, rollout_len, row_coef, **kw):
+    """Sampled-token gradient with ``row_coef[b,t]`` in place of c_t (Eq. 3; see include/adwin.h).
+    Same arguments and result as ``adwin_opd_kl_fwd_bwd`` (``grad_mode`` is fixed)."""
+    kw.pop("grad_mode", None)
+    return adwin_opd_kl_fwd_bwd(student, teacher, tokens, window, rollout_len, row_coef=row_coef,
+                                **kw)
+
+
+def adwin_return_to_go(logratio, window, rollout_len=None, gamma=0.0, flags=0, out=None):
+    """Discounted return-to-go of the per-token costs over each sequence's processed range (Eq. 3):
+    returns a [B,T] float32 tensor, zero outside the range."""
+    assert logratio.dim() == 2 and logratio.dtype == torch.float32 and logratio.is_contiguous()
+    B, T = logratio.shape
+    if out is None:
+        out = torch.empty_like(logratio)
+    _check(lib().adwin_return_to_go(_ptr(logratio), _ptr(window), _ptr(rollout_len), B, T,
+                                    float(gamma), int(flags), _ptr(out), _stream(logratio.device)))
+    return out
 
 
 def raise_on_dev_status(dev_status, allow=0):

@@ -31,6 +31,16 @@ int sm_count_of_current_device() {
   return cached[dev];
 }
 
+// Shared body of the two forward+backward entry points (row_coef is null for the plain one).
+int opd_kl_fwd_bwd_impl(const void* student_logits, const void* teacher_logits, int dtype,
+                        int64_t B, int64_t T, int64_t V, int64_t ld, const int32_t* tokens,
+                        const int32_t* window, const int32_t* rollout_len, float grad_scale,
+                        int grad_mode, int flags, void* grad_student, int grad_dtype,
+                        int64_t ld_grad, float* kl, float* logratio, float* gsq,
+                        float* lse_student, float* lse_teacher, void* workspace,
+                        size_t workspace_bytes, int32_t* dev_status, void* cuda_stream,
+                        const float* row_coef);
+
 }  // namespace
 }  // namespace adwin
 
@@ -68,6 +78,58 @@ int adwin_opd_kl_fwd_bwd(const void* student_logits, const void* teacher_logits,
                          int64_t ld_grad, float* kl, float* logratio, float* gsq,
                          float* lse_student, float* lse_teacher, void* workspace,
                          size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+  return opd_kl_fwd_bwd_impl(student_logits, teacher_logits, dtype, B, T, V, ld, tokens, window,
+                             rollout_len, grad_scale, grad_mode, flags, grad_student, grad_dtype,
+                             ld_grad, kl, logratio, gsq, lse_student, lse_teacher, workspace,
+                             workspace_bytes, dev_status, cuda_stream, nullptr);
+}
+
+int adwin_opd_kl_fwd_bwd_weighted(const void* student_logits, const void* teacher_logits,
+                                  int dtype, int64_t B, int64_t T, int64_t V, int64_t ld,
+                                  const int32_t* tokens, const int32_t* window,
+                                  const int32_t* rollout_len, const float* row_coef,
+                                  float grad_scale, int flags, void* grad_student, int grad_dtype,
+                                  int64_t ld_grad, float* kl, float* logratio, float* gsq,
+                                  float* lse_student, float* lse_teacher, void* workspace,
+                                  size_t workspace_bytes, int32_t* dev_status,
+                                  void* cuda_stream) {
+  if (B > 0 && T > 0 && !row_coef) return ADWIN_ERR_NULL;
+  if (!aligned(row_coef, 4)) return ADWIN_ERR_ALIGN;
+  return opd_kl_fwd_bwd_impl(student_logits, teacher_logits, dtype, B, T, V, ld, tokens, window,
+                             rollout_len, grad_scale, ADWIN_GRAD_SAMPLED, flags, grad_student,
+                             grad_dtype, ld_grad, kl, logratio, gsq, lse_student, lse_teacher,
+                             workspace, workspace_bytes, dev_status, cuda_stream, row_coef);
+}
+
+int adwin_return_to_go(const float* logratio, const int32_t* window, const int32_t* rollout_len,
+                       int64_t B, int64_t T, double gamma, int flags, float* rtg,
+                       void* cuda_stream) {
+  if (flags & ~ADWIN_RANGE_FULL) return ADWIN_ERR_DTYPE;
+  if (B < 0 || T < 0 || B > kMaxB || T > kMaxT) return ADWIN_ERR_SHAPE;
+  if (!(gamma >= 0.0 && gamma <= 1.0)) return ADWIN_ERR_SHAPE;
+  if (B == 0 || T == 0) return ADWIN_OK;
+  if (!logratio || !window || !rtg) return ADWIN_ERR_NULL;
+  if (!aligned(logratio, 4) || !aligned(window, 4) || !aligned(rollout_len, 4) || !aligned(rtg, 4))
+    return ADWIN_ERR_ALIGN;
+  if (launch_return_to_go(logratio, window, rollout_len, B, T, gamma, flags, rtg,
+                          static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return ADWIN_ERR_CUDA;
+  return ADWIN_OK;
+}
+
+}  // extern "C"
+
+namespace adwin {
+namespace {
+
+int opd_kl_fwd_bwd_impl(const void* student_logits, const void* teacher_logits, int dtype,
+                        int64_t B, int64_t T, int64_t V, int64_t ld, const int32_t* tokens,
+                        const int32_t* window, const int32_t* rollout_len, float grad_scale,
+                        int grad_mode, int flags, void* grad_student, int grad_dtype,
+                        int64_t ld_grad, float* kl, float* logratio, float* gsq,
+                        float* lse_student, float* lse_teacher, void* workspace,
+                        size_t workspace_bytes, int32_t* dev_status, void* cuda_stream,
+                        const float* row_coef) {
   if (dtype != ADWIN_F32 && dtype != ADWIN_BF16) return ADWIN_ERR_DTYPE;
   if (grad_mode != ADWIN_GRAD_FULL_KL && grad_mode != ADWIN_GRAD_SAMPLED) return ADWIN_ERR_DTYPE;
   if (flags & ~kKnownFlags) return ADWIN_ERR_DTYPE;
@@ -111,6 +173,7 @@ int adwin_opd_kl_fwd_bwd(const void* student_logits, const void* teacher_logits,
   p.offsets = reinterpret_cast<const int64_t*>(wbase + wl.off_offsets);
   p.range = reinterpret_cast<const int32_t*>(wbase + wl.off_range);
   p.ewin = reinterpret_cast<const int32_t*>(wbase + wl.off_ewin);
+  p.row_coef = row_coef;
 
   if (launch_rowmap(window, rollout_len, B, T, flags, workspace, kl, logratio, gsq, lse_student,
                     lse_teacher, dev_status, s) != cudaSuccess)
@@ -135,6 +198,11 @@ int adwin_opd_kl_fwd_bwd(const void* student_logits, const void* teacher_logits,
   if (launch_kl_generic(p, dtype, gd, vec16, sms, s) != cudaSuccess) return ADWIN_ERR_CUDA;
   return ADWIN_OK;
 }
+
+}  // namespace
+}  // namespace adwin
+
+extern "C" {
 
 int adwin_window_reduce(const float* kl, const float* logratio, const float* gsq,
                         const int32_t* window, const int32_t* rollout_len, int64_t B, int64_t T,

@@ -39,6 +39,9 @@ struct KlParams {
   const int32_t* range;    // [B] processed range P_b
   const int32_t* ewin;     // [B] effective window E_b
   const int64_t* offsets;  // [B+1] exclusive prefix sums of P_b
+  // SAMPLED mode only: per-position coefficient that takes the place of c_t (the discounted
+  // return-to-go of Eq. 3); null for the token-local estimator of Eq. 4
+  const float* row_coef;
 };
 
 __device__ __forceinline__ float ex2f(float x) {
@@ -172,8 +175,11 @@ struct RowScalars {
 //   KL = E_p[delta] - Delta;   c = (z_y - u_y) - Delta
 // The expanded squared norm sum p^2 (delta - E_p delta)^2 = (B2 - 2 c0 B1 + c0^2 B0) / S^2 is only
 // used for rows whose gradient is not written.
+// w: SAMPLED mode only, null or the address of a caller-supplied coefficient that takes the place
+// of c (Eq. 3); it is read only on that branch.
 __device__ __forceinline__ RowScalars finish_row(const RowTotals& t, float zy, float uy,
-                                                 bool y_valid, float dref, float alpha, int mode) {
+                                                 bool y_valid, float dref, float alpha, int mode,
+                                                 const float* w = nullptr) {
   constexpr float kLn2f = 0.69314718055994531f;
   RowScalars r;
   const float l2s = log2f(t.S), l2t = log2f(t.St);
@@ -194,7 +200,7 @@ __device__ __forceinline__ RowScalars finish_row(const RowTotals& t, float zy, f
   } else {
     const float py = y_valid ? ex2f(fmaf(zy, kLog2e, -t.M2s)) * inv_s : __int_as_float(0x7fc00000);
     const float rest = fmaxf(fmaf(t.B0, inv_s * inv_s, -py * py), 0.f);  // sum_{k != y} p_k^2
-    const float ac = alpha * r.c;
+    const float ac = alpha * (w ? *w : r.c);
     r.gsq_expanded = ac * ac * fmaf(1.f - py, 1.f - py, rest);
     r.coef = -ac * inv_s;
     r.gy = ac * (1.f - py);

@@ -40,4 +40,8 @@ cudaError_t launch_probe_align(const float* kl, const float* logratio, const flo
                                double* seq_stats, double* seq_full, double* batch_stats,
                                int32_t* L_next, int32_t* flags_out, cudaStream_t s);
 
+cudaError_t launch_return_to_go(const float* logratio, const int32_t* window,
+                                const int32_t* rollout_len, int64_t B, int64_t T, double gamma,
+                                int flags, float* rtg, cudaStream_t s);
+
 }  // namespace adwin

@@ -106,7 +106,9 @@ __global__ void __launch_bounds__(kGenericThreads) kl_generic_kernel(KlParams p)
       acc_piece<N, true>(z, u, dref, a);
     }
     const RowTotals tot = block_combine(a, sm);
-    if (tid == 0) sm.rs = finish_row(tot, zy, uy, y_valid, dref, p.alpha, p.mode);
+    if (tid == 0)
+      sm.rs = finish_row(tot, zy, uy, y_valid, dref, p.alpha, p.mode,
+                         p.row_coef ? p.row_coef + r : nullptr);
     __syncthreads();
     const RowScalars rs = sm.rs;
 

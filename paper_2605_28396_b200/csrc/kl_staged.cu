@@ -83,7 +83,8 @@ struct __align__(16) RowMeta {
   int y;
   int wg;
   float zy, uy;
-  int pad[2];
+  float w;      // caller-supplied row coefficient (0 when there is none)
+  int pad;
 };
 
 struct __align__(16) Ctrl {
@@ -640,6 +641,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       m.wg = wg ? 1 : 0;
       m.zy = zy;
       m.uy = uy;
+      m.w = p.row_coef ? p.row_coef[r] : 0.f;
       mbar_arrive(smem_u32(&ctrl.meta_full[ms]));   // release: the fields are visible
     }
   } else if (warp < kNW) {
@@ -866,7 +868,9 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       }
 
       // ---------------------------------------------------------------- row scalars
-      const RowScalars rs = finish_row(t, zyC, uyC, y_valid, dref, p.alpha, p.mode);
+      // (the row's metadata slot stays valid until this warp releases it at the end of the row)
+      const RowScalars rs = finish_row(t, zyC, uyC, y_valid, dref, p.alpha, p.mode,
+                                       p.row_coef ? &ctrl.meta[i % kMetaDepth].w : nullptr);
       if (warp == 0 && lane == 0 && rank == 0) {
         p.kl[rC] = rs.kl;
         p.logratio[rC] = rs.c;

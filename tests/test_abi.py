@@ -89,6 +89,25 @@ def test_reduce_and_align_validation(L):
                                fake, fake, fake, None) == 1
 
 
+def test_return_to_go_and_weighted_validation(L):
+    fake = ctypes.c_void_p(4096)
+    f64 = ctypes.c_double
+    assert L.adwin_return_to_go(fake, fake, None, 2, 4, f64(0.5), 0, None, None) == 1
+    assert L.adwin_return_to_go(fake, fake, None, 2, 4, f64(1.5), 0, fake, None) == 2
+    assert L.adwin_return_to_go(fake, fake, None, 2, 4, f64(-0.1), 0, fake, None) == 2
+    assert L.adwin_return_to_go(fake, fake, None, 2, 4, f64(float("nan")), 0, fake, None) == 2
+    assert L.adwin_return_to_go(fake, fake, None, 2, 4, f64(0.5), 1, fake, None) == 4
+    assert L.adwin_return_to_go(fake, fake, None, -1, 4, f64(0.5), 0, fake, None) == 2
+    assert L.adwin_return_to_go(None, None, None, 0, 4, f64(0.5), 0, None, None) == 0
+    args = [fake, fake, 1, 2, 4, 16, 16, fake, fake, None]
+    tail = [1.0, 0, None, 1, 16, fake, fake, None, None, None, fake, 1 << 20, fake, None]
+    assert L.adwin_opd_kl_fwd_bwd_weighted(*args, None, *tail) == 1       # no coefficients
+    assert L.adwin_opd_kl_fwd_bwd_weighted(*args, ctypes.c_void_p(4098), *tail) == 3
+    bad = list(tail)
+    bad[1] = 1 << 10
+    assert L.adwin_opd_kl_fwd_bwd_weighted(*args, fake, *bad) == 4        # unknown flag
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(api, "_lib", None)
     monkeypatch.setattr(api, "LIB_PATH", tmp_path / "nope.so")

@@ -7,6 +7,8 @@ calls it twice in a row through the C ABI, with different windows, shapes and gr
 that a second call that reused anything the first one left in that array would be caught, and
 compares every output with ``adwin_opd_kl_fwd_bwd`` on the same inputs.
 """
+import gc
+
 import pytest
 import torch
 
@@ -27,6 +29,7 @@ def _both(batch, mode, flags, grad_dtype):
     grad = torch.full((B, T, V), 3.0, dtype=grad_dtype, device=DEV)
     kl, c, q = (torch.full((B, T), -1.0, **f32) for _ in range(3))
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    gc.collect()   # tensors that earlier tests left in reference cycles must not be freed midway
     torch.cuda.synchronize()
     before = torch.cuda.memory_allocated(DEV)
     api.adwin_opd_kl_fwd_bwd_no_alloc(batch.student, batch.teacher, batch.tokens, batch.window,
