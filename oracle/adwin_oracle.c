@@ -390,6 +390,47 @@ void adwin_oracle_row_weighted(const double *z, int64_t V, int64_t y, double alp
   *gsq = q2 + q2c;
 }
 
+/*
+ * Teacher-side drift of one position (Section 3.1): the entropy of the teacher distribution
+ * q = softmax(u), H = - sum_k q_k log q_k (0 log 0 = 0), whose exponential is the teacher
+ * branching factor BF, and the rank of the sampled token under q: 1 + the number of entries with a
+ * strictly larger logit.  y outside [0,V) gives rank 0.
+ */
+void adwin_oracle_teacher_drift_row(const double *u, int64_t V, int64_t y, double *entropy,
+                                    int64_t *rank) {
+  double lt = adwin_oracle_logsumexp(u, V);
+  double acc = 0.0, comp = 0.0;
+  int64_t above = 0;
+  for (int64_t k = 0; k < V; ++k) {
+    double lq = u[k] - lt;
+    double q = exp(lq);
+    if (q != 0.0) comp_add(&acc, &comp, -q * lq);
+    if (y >= 0 && y < V && u[k] > u[y]) ++above;
+  }
+  *entropy = acc + comp;
+  *rank = (y >= 0 && y < V) ? above + 1 : 0;
+}
+
+/*
+ * The survival fraction S_T^(k) of Section 3.1, literally: for every position T' (0-based) the
+ * fraction of the B rollouts in which every position t <= T' that belongs to the rollout
+ * (t < R_b) has rank <= k.  rank is [B,T] (entries past the rollout are ignored).
+ */
+void adwin_oracle_topk_survival(const int64_t *rank, const int32_t *rollout_len, int64_t B,
+                                int64_t T, int64_t k, double *survival) {
+  for (int64_t tp = 0; tp < T; ++tp) {
+    int64_t alive = 0;
+    for (int64_t b = 0; b < B; ++b) {
+      int64_t R = rollout_len ? rollout_len[b] : T;
+      int ok = 1;
+      for (int64_t t = 0; t <= tp && t < R; ++t)
+        if (rank[b * T + t] > k) ok = 0;
+      alive += ok;
+    }
+    survival[tp] = (double)alive / (double)B;
+  }
+}
+
 int adwin_oracle_num_threads(void) {
 #ifdef _OPENMP
   extern int omp_get_max_threads(void);

@@ -194,3 +194,24 @@ def row_weighted(z, y: int, alpha: float, w: float):
                                     ctypes.c_double(alpha), ctypes.c_double(w), ctypes.byref(gsq),
                                     _p(g))
     return g, gsq.value
+
+
+def teacher_drift_row(u, y: int):
+    """Entropy (nats) of softmax(u) and the rank of token y under it (Section 3.1)."""
+    u = _f64(u)
+    H = ctypes.c_double()
+    r = ctypes.c_int64()
+    lib().adwin_oracle_teacher_drift_row(_p(u), ctypes.c_int64(u.size), ctypes.c_int64(int(y)),
+                                         ctypes.byref(H), ctypes.byref(r))
+    return H.value, int(r.value)
+
+
+def topk_survival(rank, rollout_len, k: int):
+    """S_T^(k) for every position T: [T] float64 (Section 3.1)."""
+    rank = np.ascontiguousarray(rank, dtype=np.int64)
+    B, T = rank.shape
+    rollout_len = _i32(rollout_len)
+    out = np.empty(T, dtype=np.float64)
+    lib().adwin_oracle_topk_survival(_p(rank), _p(rollout_len), ctypes.c_int64(B),
+                                     ctypes.c_int64(T), ctypes.c_int64(int(k)), _p(out))
+    return out
