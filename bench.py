@@ -305,6 +305,75 @@ def run_ours(args):
     ms_step = ms_total / args.steps
     value = rows_all / (ms_step / 1e3)
 
+    # ---- the two-pass update with return-to-go weights (Eq. 3, gamma > 0), same batch: a read-only
+    # pass for the costs, the scan over [B,T], the sampled-token gradient pass with the weights
+    rtg_line = None
+    if rank == 0 and world == 1:
+        gamma, n_rtg = 0.9, 5
+        probe = rtg = wout = None
+
+        def rtg_step():
+            nonlocal probe, rtg, wout
+            probe = api.adwin_opd_kl_fwd_bwd(batch.student, batch.teacher, batch.tokens,
+                                             batch.window, batch.rollout_len, out=probe,
+                                             workspace=ws, dev_status=status)
+            rtg = api.adwin_return_to_go(probe.logratio, batch.window, batch.rollout_len, gamma,
+                                         out=rtg)
+            wout = api.adwin_opd_kl_fwd_bwd_weighted(batch.student, batch.teacher, batch.tokens,
+                                                     batch.window, batch.rollout_len, rtg,
+                                                     grad=grad, out=wout, workspace=ws,
+                                                     dev_status=status)
+        for _ in range(3):
+            rtg_step()
+        torch.cuda.synchronize()
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        r0.record()
+        for _ in range(n_rtg):
+            rtg_step()
+        r1.record()
+        torch.cuda.synchronize()
+        rms = r0.elapsed_time(r1) / n_rtg
+        rbytes = rows * V * 10          # 2 reads (pass 1) + 2 reads and 1 write (pass 2), bf16
+        rtg_line = {"gamma": gamma, "ms_per_step": rms, "tokens_per_s": rows / (rms / 1e3),
+                    "algorithmic_bytes": rbytes, "achieved_gbs": rbytes / (rms * 1e-3) / 1e9,
+                    "launches_per_step": 2 * 2 + 1, "steps": n_rtg,
+                    "path": "adwin_opd_kl_fwd_bwd (no gradient) -> adwin_return_to_go -> "
+                            "adwin_opd_kl_fwd_bwd_weighted"}
+        if int(status.item()):
+            raise SystemExit("device status set by the return-to-go path")
+
+    # ---- teacher-drift diagnostics (Section 3.1) over every position of the same batch: one read
+    # of the teacher logits, then the survival / branching-factor curves
+    drift_line = None
+    if rank == 0 and world == 1:
+        n_drift = 5
+        ks = torch.tensor([1, 5, 20], dtype=torch.int32, device=dev)
+
+        def drift_step():
+            d = api.adwin_teacher_drift(batch.teacher, batch.tokens, batch.rollout_len,
+                                        dev_status=status)
+            return api.adwin_drift_curves(d.entropy, d.rank, batch.rollout_len, ks)
+        for _ in range(3):
+            drift_step()
+        torch.cuda.synchronize()
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record()
+        for _ in range(n_drift):
+            drift_step()
+        d1.record()
+        torch.cuda.synchronize()
+        dms = d0.elapsed_time(d1) / n_drift
+        drows = int(batch.rollout_len.sum())
+        dbytes = drows * V * 2          # every teacher logit once
+        peak_d, _ = measured_peak()
+        drift_line = {"ms_per_step": dms, "positions": drows, "tokens_per_s": drows / (dms / 1e3),
+                      "algorithmic_bytes": dbytes, "achieved_gbs": dbytes / (dms * 1e-3) / 1e9,
+                      "frac_of_measured_peak": dbytes / (dms * 1e-3) / 1e9 / peak_d,
+                      "launches_per_step": 3, "steps": n_drift,
+                      "path": "adwin_teacher_drift -> adwin_drift_curves (timed together)"}
+        if int(status.item()):
+            raise SystemExit("device status set by the teacher-drift path")
+
     # ---- end to end through the host-buffer entry point (copies inside the timed region)
     e2e = None
     if not args.no_e2e:
@@ -374,7 +443,8 @@ def run_ours(args):
                      "kernel_ms": kernel_ms, "algorithmic_bytes": alg_bytes,
                      "frac_of_nominal_8TBps": achieved / 8000.0},
         "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": LAUNCHES_PER_STEP * args.steps,
-        "clocks": clocks, "windowed_kl_sum": loss,
+        "clocks": clocks, "windowed_kl_sum": loss, "return_to_go_path": rtg_line,
+        "teacher_drift_path": drift_line,
         "L_next": int(al.L_next.item()),
     }
     print(json.dumps(line))

@@ -194,6 +194,38 @@ int adwin_opd_kl_fwd_bwd_weighted(const void* student_logits, const void* teache
                                   size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
 
 /*
+ * Teacher-side drift along student rollouts (Section 3.1), one read of the teacher logits:
+ *   entropy[b,t] = H[softmax(teacher_logits[b,t,:])] in nats; the teacher branching factor
+ *                  (per-position perplexity) is BF = exp(entropy);
+ *   rank[b,t]    = rank r of the sampled token tokens[b,t] under the teacher distribution,
+ *                  1 + the number of vocabulary entries whose logit is strictly larger (equal
+ *                  logits share the better rank); int32.
+ * Positions t < R_b are processed (rollout_len NULL => T), the others get entropy 0 and rank 0.
+ * Pointers, dtype, strides and dev_status as in adwin_opd_kl_fwd_bwd (no workspace is needed);
+ * a token outside [0,V) gives rank 0 and ADWIN_DEV_TOKEN_RANGE, a non-finite entropy
+ * ADWIN_DEV_NONFINITE, an invalid R_b is clamped and raises ADWIN_DEV_WINDOW.
+ */
+int adwin_teacher_drift(const void* teacher_logits, int dtype, int64_t B, int64_t T, int64_t V,
+                        int64_t ld, const int32_t* tokens, const int32_t* rollout_len,
+                        float* entropy, int32_t* rank, int32_t* dev_status, void* cuda_stream);
+
+/*
+ * The two curves of Section 3.1 over the B rollouts of a batch, per position t:
+ *   worst_rank[b,t] = max_{t' <= t} rank[b,t']      [B,T] int32 (a rollout that has ended keeps
+ *                     its value: it collects no further rejections);
+ *   survival[j,t]   = (1/B) * #{b : worst_rank[b,t] <= ks[j]} = S_t^(k) for k = ks[j], the
+ *                     fraction of rollouts with no top-k rejection through position t
+ *                     (cumulative rejection is 1 - survival);   [K,T] float64, 0 <= K <= 64;
+ *   bf_mean[t]      = mean of exp(entropy[b,t]) over the rollouts still running at t (t < R_b),
+ *                     0 where none is;   [T] float64;        n_active[t] = their number, [T] int32.
+ * entropy, rank: the outputs of adwin_teacher_drift.  ks: [K] int32 DEVICE pointer.  All pointers
+ * are device pointers; sums run over the sequences in index order.
+ */
+int adwin_drift_curves(const float* entropy, const int32_t* rank, const int32_t* rollout_len,
+                       int64_t B, int64_t T, const int32_t* ks, int32_t K, int32_t* worst_rank,
+                       double* survival, double* bf_mean, int32_t* n_active, void* cuda_stream);
+
+/*
  * The same pass for logits that live in HOST memory (pinned memory gives asynchronous copies).
  * Only the rows inside the processed range cross PCIe -- the window skip of Section 4.1 saves the
  * transfer as well as the arithmetic -- in stages of at most rows_per_stage rows of one sequence;

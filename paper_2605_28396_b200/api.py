@@ -28,7 +28,8 @@ EXPORTS = ("adwin_version", "adwin_status_string", "adwin_workspace_bytes",
            "adwin_opd_kl_fwd_bwd", "adwin_window_reduce", "adwin_probe_align",
            "adwin_host_staging_bytes", "adwin_opd_kl_fwd_bwd_host",
            "adwin_no_alloc_max_sequences", "adwin_opd_kl_fwd_bwd_no_alloc",
-           "adwin_return_to_go", "adwin_opd_kl_fwd_bwd_weighted")
+           "adwin_return_to_go", "adwin_opd_kl_fwd_bwd_weighted", "adwin_teacher_drift",
+           "adwin_drift_curves")
 
 _lib = None
 
@@ -82,6 +83,11 @@ def lib():
                                                     vp, vp, vp, f32, ctypes.c_int, vp,
                                                     ctypes.c_int, i64, vp, vp, vp, vp, vp, vp, sz,
                                                     vp, vp]
+        L.adwin_teacher_drift.restype = ctypes.c_int
+        L.adwin_teacher_drift.argtypes = [vp, ctypes.c_int, i64, i64, i64, i64, vp, vp, vp, vp, vp,
+                                          vp]
+        L.adwin_drift_curves.restype = ctypes.c_int
+        L.adwin_drift_curves.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -302,3 +308,42 @@ def adwin_opd_kl_fwd_bwd_no_alloc(student, teacher, tokens, window, rollout_len,
         _ptr(window), _ptr(rollout_len), float(grad_scale), int(grad_mode), int(flags), _ptr(grad),
         _dtype_code(grad.dtype) if grad is not None else 0, ld_grad, _ptr(kl), _ptr(logratio),
         _ptr(gsq), _ptr(lse_s), _ptr(lse_t), _ptr(dev_status), _stream(student.device)))
+
+
+def adwin_teacher_drift(teacher, tokens, rollout_len=None, dev_status=None):
+    """Teacher entropy (nats) and rank of the sampled token per position (Section 3.1).
+    Returns a namespace with entropy [B,T] float32, rank [B,T] int32, dev_status."""
+    assert teacher.is_cuda and teacher.dim() == 3
+    B, T, V = teacher.shape
+    dev = teacher.device
+    assert teacher.stride(2) == 1 or V == 1, "last dim must be contiguous"
+    ld = teacher.stride(1) if T > 1 else (teacher.stride(0) if B > 1 else V)
+    assert B <= 1 or T <= 1 or teacher.stride(0) == T * ld, "rows must sit at one uniform stride"
+    o = SimpleNamespace()
+    o.entropy = torch.empty((B, T), dtype=torch.float32, device=dev)
+    o.rank = torch.empty((B, T), dtype=torch.int32, device=dev)
+    o.dev_status = dev_status if dev_status is not None else torch.zeros(1, dtype=torch.int32,
+                                                                         device=dev)
+    _check(lib().adwin_teacher_drift(_ptr(teacher), _dtype_code(teacher.dtype), B, T, V, ld,
+                                     _ptr(tokens), _ptr(rollout_len), _ptr(o.entropy),
+                                     _ptr(o.rank), _ptr(o.dev_status), _stream(dev)))
+    return o
+
+
+def adwin_drift_curves(entropy, rank, rollout_len=None, ks=(1, 5, 20)):
+    """Top-k survival and mean branching factor per position over the batch (Section 3.1).
+    Returns a namespace with worst_rank [B,T] int32, survival [K,T] float64, bf_mean [T] float64,
+    n_active [T] int32."""
+    B, T = entropy.shape
+    dev = entropy.device
+    ks_t = ks if torch.is_tensor(ks) else torch.tensor(list(ks), dtype=torch.int32, device=dev)
+    K = int(ks_t.numel())
+    o = SimpleNamespace()
+    o.worst_rank = torch.empty((B, T), dtype=torch.int32, device=dev)
+    o.survival = torch.empty((K, T), dtype=torch.float64, device=dev)
+    o.bf_mean = torch.empty(T, dtype=torch.float64, device=dev)
+    o.n_active = torch.empty(T, dtype=torch.int32, device=dev)
+    _check(lib().adwin_drift_curves(_ptr(entropy), _ptr(rank), _ptr(rollout_len), B, T,
+                                    _ptr(ks_t), K, _ptr(o.worst_rank), _ptr(o.survival),
+                                    _ptr(o.bf_mean), _ptr(o.n_active), _stream(dev)))
+    return o

@@ -117,6 +117,46 @@ int adwin_return_to_go(const float* logratio, const int32_t* window, const int32
   return ADWIN_OK;
 }
 
+int adwin_teacher_drift(const void* teacher_logits, int dtype, int64_t B, int64_t T, int64_t V,
+                        int64_t ld, const int32_t* tokens, const int32_t* rollout_len,
+                        float* entropy, int32_t* rank, int32_t* dev_status, void* cuda_stream) {
+  if (dtype != ADWIN_F32 && dtype != ADWIN_BF16) return ADWIN_ERR_DTYPE;
+  if (B < 0 || T < 0 || B > kMaxB || T > kMaxT || V < 1 || V > kMaxV || ld < V)
+    return ADWIN_ERR_SHAPE;
+  if (!dev_status) return ADWIN_ERR_NULL;
+  if (B == 0 || T == 0) return ADWIN_OK;
+  if (!teacher_logits || !tokens || !entropy || !rank) return ADWIN_ERR_NULL;
+  const size_t es = elem_size(dtype);
+  if (!aligned(teacher_logits, es) || !aligned(tokens, 4) || !aligned(rollout_len, 4) ||
+      !aligned(entropy, 4) || !aligned(rank, 4) || !aligned(dev_status, 4))
+    return ADWIN_ERR_ALIGN;
+  const int sms = sm_count_of_current_device();
+  if (sms <= 0) return ADWIN_ERR_CUDA;
+  const bool vec16 = aligned(teacher_logits, 16) && (ld * es) % 16 == 0 && (V * es) % 16 == 0;
+  if (launch_teacher_drift(teacher_logits, dtype, B, T, V, ld, tokens, rollout_len, entropy, rank,
+                           dev_status, vec16, sms,
+                           static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return ADWIN_ERR_CUDA;
+  return ADWIN_OK;
+}
+
+int adwin_drift_curves(const float* entropy, const int32_t* rank, const int32_t* rollout_len,
+                       int64_t B, int64_t T, const int32_t* ks, int32_t K, int32_t* worst_rank,
+                       double* survival, double* bf_mean, int32_t* n_active, void* cuda_stream) {
+  if (B < 0 || T < 0 || B > kMaxB || T > kMaxT || K < 0 || K > 64) return ADWIN_ERR_SHAPE;
+  if (B == 0 || T == 0) return ADWIN_OK;
+  if (!entropy || !rank || !worst_rank || !bf_mean || !n_active) return ADWIN_ERR_NULL;
+  if (K > 0 && (!ks || !survival)) return ADWIN_ERR_NULL;
+  if (!aligned(entropy, 4) || !aligned(rank, 4) || !aligned(rollout_len, 4) || !aligned(ks, 4) ||
+      !aligned(worst_rank, 4) || !aligned(survival, 8) || !aligned(bf_mean, 8) ||
+      !aligned(n_active, 4))
+    return ADWIN_ERR_ALIGN;
+  if (launch_drift_curves(entropy, rank, rollout_len, B, T, ks, K, worst_rank, survival, bf_mean,
+                          n_active, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return ADWIN_ERR_CUDA;
+  return ADWIN_OK;
+}
+
 }  // extern "C"
 
 namespace adwin {

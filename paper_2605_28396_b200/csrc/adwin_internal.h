@@ -44,4 +44,14 @@ cudaError_t launch_return_to_go(const float* logratio, const int32_t* window,
                                 const int32_t* rollout_len, int64_t B, int64_t T, double gamma,
                                 int flags, float* rtg, cudaStream_t s);
 
+cudaError_t launch_teacher_drift(const void* teacher, int dtype, int64_t B, int64_t T, int64_t V,
+                                 int64_t ld, const int32_t* tokens, const int32_t* rollout_len,
+                                 float* entropy, int32_t* rank, int32_t* status, bool vec,
+                                 int sm_count, cudaStream_t s);
+
+cudaError_t launch_drift_curves(const float* entropy, const int32_t* rank,
+                                const int32_t* rollout_len, int64_t B, int64_t T,
+                                const int32_t* ks, int32_t K, int32_t* worst, double* survival,
+                                double* bf_mean, int32_t* n_active, cudaStream_t s);
+
 }  // namespace adwin

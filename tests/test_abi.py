@@ -108,6 +108,21 @@ def test_return_to_go_and_weighted_validation(L):
     assert L.adwin_opd_kl_fwd_bwd_weighted(*args, fake, *bad) == 4        # unknown flag
 
 
+def test_drift_validation(L):
+    fake = ctypes.c_void_p(4096)
+    assert L.adwin_teacher_drift(fake, 7, 2, 4, 16, 16, fake, None, fake, fake, fake, None) == 4
+    assert L.adwin_teacher_drift(fake, 1, 2, 4, 16, 8, fake, None, fake, fake, fake, None) == 2
+    assert L.adwin_teacher_drift(fake, 1, 2, 4, 16, 16, fake, None, None, fake, fake, None) == 1
+    assert L.adwin_teacher_drift(fake, 1, 2, 4, 16, 16, fake, None, fake, fake, None, None) == 1
+    assert L.adwin_teacher_drift(ctypes.c_void_p(4097), 1, 2, 4, 16, 16, fake, None, fake, fake,
+                                 fake, None) == 3
+    assert L.adwin_teacher_drift(None, 1, 0, 4, 16, 16, None, None, None, None, fake, None) == 0
+    assert L.adwin_drift_curves(fake, fake, None, 2, 4, fake, 65, fake, fake, fake, fake, None) == 2
+    assert L.adwin_drift_curves(fake, fake, None, 2, 4, None, 2, fake, fake, fake, fake, None) == 1
+    assert L.adwin_drift_curves(fake, fake, None, 2, 4, fake, 2, None, fake, fake, fake, None) == 1
+    assert L.adwin_drift_curves(None, None, None, 0, 4, None, 0, None, None, None, None, None) == 0
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(api, "_lib", None)
     monkeypatch.setattr(api, "LIB_PATH", tmp_path / "nope.so")
