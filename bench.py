@@ -342,6 +342,42 @@ def run_ours(args):
         if int(status.item()):
             raise SystemExit("device status set by the return-to-go path")
 
+    # ---- the delayed full-rollout probe (Section 4.2) on the same batch: every position t < R_b,
+    # read-only, followed by the audit; this is the pass that config 4 runs at T = 8192
+    probe_line = None
+    if rank == 0 and world == 1:
+        n_probe = 5
+        pout = None
+
+        def probe_step():
+            nonlocal pout
+            pout = api.adwin_opd_kl_fwd_bwd(batch.student, batch.teacher, batch.tokens,
+                                            batch.window, batch.rollout_len, out=pout,
+                                            flags=api.RANGE_FULL, workspace=ws, dev_status=status)
+            return api.adwin_probe_align(pout.kl, pout.logratio, pout.gsq, batch.window,
+                                         batch.rollout_len)
+        for _ in range(3):
+            probe_step()
+        torch.cuda.synchronize()
+        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        q0.record()
+        for _ in range(n_probe):
+            probe_step()
+        q1.record()
+        torch.cuda.synchronize()
+        pms = q0.elapsed_time(q1) / n_probe
+        prows = int(batch.rollout_len.sum())
+        pbytes = prows * V * 4          # student and teacher logits once each, bf16
+        peak_p, _ = measured_peak()
+        probe_line = {"ms_per_step": pms, "positions": prows, "tokens_per_s": prows / (pms / 1e3),
+                      "algorithmic_bytes": pbytes, "achieved_gbs": pbytes / (pms * 1e-3) / 1e9,
+                      "frac_of_measured_peak": pbytes / (pms * 1e-3) / 1e9 / peak_p,
+                      "launches_per_step": 2 + 3, "steps": n_probe,
+                      "path": "adwin_opd_kl_fwd_bwd (RANGE_FULL, no gradient: kl_generic_kernel) "
+                              "-> adwin_probe_align (timed together)"}
+        if int(status.item()):
+            raise SystemExit("device status set by the probe pass")
+
     # ---- teacher-drift diagnostics (Section 3.1) over every position of the same batch: one read
     # of the teacher logits, then the survival / branching-factor curves
     drift_line = None
@@ -443,7 +479,7 @@ def run_ours(args):
                      "kernel_ms": kernel_ms, "algorithmic_bytes": alg_bytes,
                      "frac_of_nominal_8TBps": achieved / 8000.0},
         "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": LAUNCHES_PER_STEP * args.steps,
-        "clocks": clocks, "windowed_kl_sum": loss, "return_to_go_path": rtg_line,
+        "clocks": clocks, "windowed_kl_sum": loss, "probe_pass": probe_line, "return_to_go_path": rtg_line,
         "teacher_drift_path": drift_line,
         "L_next": int(al.L_next.item()),
     }

@@ -65,7 +65,10 @@ enum {
   ADWIN_ZERO_TAIL = 1,     /* zero-fill gradient rows t >= E_b instead of leaving them untouched */
   ADWIN_RANGE_FULL = 2,    /* per-token scalars for every t < R_b (delayed full-rollout probe,
                               Section 4.2); the gradient is still written only for t < E_b */
-  ADWIN_FORCE_GENERIC = 4  /* use the shape-agnostic kernel even when the staged kernel applies */
+  ADWIN_FORCE_GENERIC = 4, /* use the row-per-CTA streaming kernel for every row */
+  ADWIN_FORCE_STAGED = 8   /* use the staged cluster kernel wherever the 16-byte layout allows,
+                              also for calls without gradient (which by default go to the
+                              streaming kernel: one sweep, nothing to keep on chip) */
 };
 
 /* Flags returned by adwin_probe_align in *flags_out. */

@@ -18,7 +18,7 @@ LIB_PATH = _PKG / "libadwin_b200.so"
 OK = 0
 F32, BF16 = 0, 1
 GRAD_FULL_KL, GRAD_SAMPLED = 0, 1
-ZERO_TAIL, RANGE_FULL, FORCE_GENERIC = 1, 2, 4
+ZERO_TAIL, RANGE_FULL, FORCE_GENERIC, FORCE_STAGED = 1, 2, 4, 8
 DEV_TOKEN_RANGE, DEV_NONFINITE, DEV_TIMEOUT, DEV_BOUNDS, DEV_WINDOW = 1, 2, 4, 8, 16
 ALIGN_DEGENERATE, ALIGN_NONE_ADMISSIBLE = 1, 2
 DEFAULT_CANDIDATES = (64, 128, 256, 512, 1024, 2048)   # Section 5.1, Training Details

@@ -62,6 +62,7 @@ def test_host_side_argument_validation(L):
     assert _call(L, dtype=7) == 4
     assert _call(L, mode=2) == 4
     assert _call(L, flags=1 << 10) == 4
+    assert _call(L, flags=16) == 4
     assert _call(L, V=0) == 2
     assert _call(L, ld=8) == 2
     assert _call(L, B=-1) == 2

@@ -11,7 +11,7 @@ from tests import parity as P
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
-PATHS = {"staged": 0, "generic": api.FORCE_GENERIC}
+PATHS = {"staged": api.FORCE_STAGED, "generic": api.FORCE_GENERIC, "default": 0}
 
 
 def run_and_check(batch, *, grad_dtype, grad_mode=api.GRAD_FULL_KL, flags=0, grad_scale=1.0,

@@ -12,7 +12,7 @@ from tests import parity as P
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
-PATHS = {"staged": 0, "generic": api.FORCE_GENERIC}
+PATHS = {"staged": api.FORCE_STAGED, "generic": api.FORCE_GENERIC, "default": 0}
 
 
 def _check_rtg(got, c64, window, rollout, gamma, flags):
