@@ -62,8 +62,8 @@ def measured_peak():
 
 # DRAM bytes per processed row of the staged kernel, from the committed ncu capture
 # (profiles/kl_staged_bf16_small_case_full.md), valid for the kernel source with this fingerprint.
-TRAFFIC_BYTES_PER_ROW = 856533
-TRAFFIC_KERNEL_SHA = "d431a86876ebb815"
+TRAFFIC_BYTES_PER_ROW = 856860
+TRAFFIC_KERNEL_SHA = "f589595c7073be11"
 
 
 def recorded_traffic(rows):
