@@ -84,8 +84,11 @@ int adwin_version(void);
 const char* adwin_status_string(int status);
 
 /*
- * Bytes of device scratch that adwin_opd_kl_fwd_bwd needs for these shapes (the in-window row map:
- * effective ranges and their prefix sums).  Always > 0; the buffer must be 256-byte aligned.
+ * Bytes of device scratch that adwin_opd_kl_fwd_bwd wants for these shapes (the row map:
+ * effective ranges and two sets of prefix sums, about 24 bytes per sequence).  Always > 0; the
+ * buffer must be 256-byte aligned.  A buffer that holds only the first set (about two thirds of
+ * this size) is still accepted: the call then runs an ADWIN_RANGE_FULL request with gradient as
+ * one kernel instead of two, with the same results to within rounding.
  */
 size_t adwin_workspace_bytes(int64_t B, int64_t T, int64_t V, int dtype, int flags);
 

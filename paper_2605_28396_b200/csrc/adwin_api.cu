@@ -69,7 +69,7 @@ const char* adwin_status_string(int status) {
 size_t adwin_workspace_bytes(int64_t B, int64_t T, int64_t V, int dtype, int flags) {
   (void)T; (void)V; (void)dtype; (void)flags;
   if (B < 0) B = 0;
-  return workspace_layout(B).total;
+  return workspace_layout(B).total_ext;
 }
 
 int adwin_opd_kl_fwd_bwd(const void* student_logits, const void* teacher_logits, int dtype,
@@ -190,7 +190,7 @@ int opd_kl_fwd_bwd_impl(const void* student_logits, const void* teacher_logits, 
     return ADWIN_ERR_ALIGN;
   if (grad_student && !aligned(grad_student, elem_size(grad_dtype))) return ADWIN_ERR_ALIGN;
   if (!workspace || !aligned(workspace, 256) ||
-      workspace_bytes < adwin_workspace_bytes(B, T, V, dtype, flags))
+      workspace_bytes < workspace_layout(B).total)
     return ADWIN_ERR_WORKSPACE;
   const int sms = sm_count_of_current_device();
   if (sms <= 0) return ADWIN_ERR_CUDA;
@@ -215,22 +215,44 @@ int opd_kl_fwd_bwd_impl(const void* student_logits, const void* teacher_logits, 
   p.range = reinterpret_cast<const int32_t*>(wbase + wl.off_range);
   p.ewin = reinterpret_cast<const int32_t*>(wbase + wl.off_ewin);
   p.row_coef = row_coef;
+  p.skip_below = nullptr;
 
-  if (launch_rowmap(window, rollout_len, B, T, flags, workspace, kl, logratio, gsq, lse_student,
-                    lse_teacher, dev_status, s) != cudaSuccess)
-    return ADWIN_ERR_CUDA;
-  if ((flags & ADWIN_ZERO_TAIL) && grad_student) {
-    if (launch_zero_tail(p, grad_dtype, s) != cudaSuccess) return ADWIN_ERR_CUDA;
-  }
-
-  // 16-byte layout test shared by the vectorised generic path and the staged kernel.
+  // 16-byte layout test shared by the vectorised streaming path and the staged kernel.
   const int gd = grad_student ? grad_dtype : dtype;
   bool vec16 = aligned(student_logits, 16) && aligned(teacher_logits, 16) &&
                (ld * es) % 16 == 0 && (V * es) % 16 == 0;
   if (grad_student)
     vec16 = vec16 && aligned(grad_student, 16) && (ld_grad * elem_size(gd)) % 16 == 0 &&
             (V * elem_size(gd)) % 16 == 0;
+  // Scalars over the whole rollout with the gradient inside the window: the window rows need the
+  // staged kernel's two sweeps, the rows past the window are a single read, which the streaming
+  // kernel does faster.  With the extended workspace the call runs them as two launches.
+  const bool split = vec16 && grad_student && (flags & ADWIN_RANGE_FULL) &&
+                     !(flags & (ADWIN_FORCE_GENERIC | ADWIN_FORCE_STAGED)) &&
+                     workspace_bytes >= wl.total_ext;
 
+  if (launch_rowmap(window, rollout_len, B, T, flags, workspace, split, kl, logratio, gsq,
+                    lse_student, lse_teacher, dev_status, s) != cudaSuccess)
+    return ADWIN_ERR_CUDA;
+  if ((flags & ADWIN_ZERO_TAIL) && grad_student) {
+    if (launch_zero_tail(p, grad_dtype, s) != cudaSuccess) return ADWIN_ERR_CUDA;
+  }
+
+  if (split) {
+    KlParams pw = p;          // window rows: the compact list built from the effective windows
+    pw.offsets = reinterpret_cast<const int64_t*>(wbase + wl.off_offsets_win);
+    pw.range = p.ewin;
+    const cudaError_t e = launch_kl_staged(pw, dtype, gd, sms, s);
+    if (e == cudaSuccess) {
+      KlParams pr = p;        // the rest of every rollout, without gradient
+      pr.grad = nullptr;
+      pr.ld_grad = 0;
+      pr.skip_below = p.ewin;
+      if (launch_kl_generic(pr, dtype, dtype, true, sms, s) != cudaSuccess) return ADWIN_ERR_CUDA;
+      return ADWIN_OK;
+    }
+    if (e != cudaErrorNotSupported) return ADWIN_ERR_CUDA;
+  }
   // Rows whose gradient is written need two sweeps with the row kept on chip in between: the
   // staged cluster kernel.  A call without gradient is a single read of every row, which the
   // row-per-CTA streaming kernel does faster (90 % against 74 % of the copy bandwidth, measured).

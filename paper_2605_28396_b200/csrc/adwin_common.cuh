@@ -42,6 +42,8 @@ struct KlParams {
   // SAMPLED mode only: per-position coefficient that takes the place of c_t (the discounted
   // return-to-go of Eq. 3); null for the token-local estimator of Eq. 4
   const float* row_coef;
+  // streaming kernel only: when set, positions t < skip_below[b] are left to another launch
+  const int32_t* skip_below;
 };
 
 __device__ __forceinline__ float ex2f(float x) {

@@ -10,15 +10,20 @@ namespace adwin {
 
 struct KlParams;
 
-// Workspace layout: [0,256) reserved counters; offsets (B+1) int64; range B int32; ewin B int32.
+// Workspace layout: [0,256) reserved counters; offsets (B+1) int64; range B int32; ewin B int32:
+// `total` bytes, the part every call needs.  Optional extension up to `total_ext`: a second
+// prefix-sum array over the effective windows, offsets_win (B+1) int64, which lets a call that
+// wants scalars over the rollout and the gradient inside the window run as two kernels.
 struct WorkspaceLayout {
   size_t off_offsets, off_range, off_ewin, total;
+  size_t off_offsets_win, total_ext;
 };
 WorkspaceLayout workspace_layout(int64_t B);
 
 cudaError_t launch_rowmap(const int32_t* window, const int32_t* rollout_len, int64_t B, int64_t T,
-                          int flags, void* workspace, float* kl, float* logratio, float* gsq,
-                          float* lse_s, float* lse_t, int32_t* status, cudaStream_t s);
+                          int flags, void* workspace, bool with_window_offsets, float* kl,
+                          float* logratio, float* gsq, float* lse_s, float* lse_t, int32_t* status,
+                          cudaStream_t s);
 
 cudaError_t launch_zero_tail(const KlParams& p, int grad_dtype, cudaStream_t s);
 

@@ -84,6 +84,7 @@ __global__ void __launch_bounds__(kGenericThreads) kl_generic_kernel(KlParams p)
     const int64_t b = r / p.T;
     const int t = (int)(r - b * p.T);
     if (t >= p.range[b]) continue;  // past the window: the row is never touched
+    if (p.skip_below && t < p.skip_below[b]) continue;
     const bool write_grad = (p.grad != nullptr) && (t < p.ewin[b]);
 
     const char* zrow = static_cast<const char*>(p.student) + (size_t)r * p.ld * sizeof(TIn);

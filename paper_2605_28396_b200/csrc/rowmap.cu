@@ -17,6 +17,8 @@ WorkspaceLayout workspace_layout(int64_t B) {
   w.off_range = up(w.off_offsets + (size_t)(B + 1) * sizeof(int64_t));
   w.off_ewin = up(w.off_range + (size_t)B * sizeof(int32_t));
   w.total = up(w.off_ewin + (size_t)B * sizeof(int32_t));
+  w.off_offsets_win = w.total;
+  w.total_ext = up(w.off_offsets_win + (size_t)(B + 1) * sizeof(int64_t));
   return w;
 }
 
@@ -34,14 +36,14 @@ __device__ __forceinline__ void clamp_lengths(int32_t w, int32_t r, int64_t T, i
 // Block 0: scan.  Blocks >= 1: zero the per-token outputs of rows outside the processed range.
 __global__ void __launch_bounds__(kMapThreads) rowmap_kernel(
     const int32_t* __restrict__ window, const int32_t* __restrict__ rollout_len, int64_t B,
-    int64_t T, int flags, int64_t* offsets, int32_t* range, int32_t* ewin, float* kl,
-    float* logratio, float* gsq, float* lse_s, float* lse_t, int32_t* status) {
+    int64_t T, int flags, int64_t* offsets, int64_t* offsets_win, int32_t* range, int32_t* ewin,
+    float* kl, float* logratio, float* gsq, float* lse_s, float* lse_t, int32_t* status) {
   if (blockIdx.x == 0) {
     __shared__ int64_t part[kMapThreads];
     const int tid = threadIdx.x;
     const int64_t per = (B + kMapThreads - 1) / kMapThreads;
     const int64_t b0 = tid * per, b1 = (b0 + per < B) ? b0 + per : B;
-    int64_t sum = 0;
+    int64_t sum = 0, sum_win = 0;
     bool any_bad = false;
     for (int64_t b = b0; b < b1; ++b) {
       int E, P;
@@ -51,6 +53,7 @@ __global__ void __launch_bounds__(kMapThreads) rowmap_kernel(
       range[b] = P;
       ewin[b] = E;
       sum += P;
+      sum_win += E;
     }
     part[tid] = sum;
     __syncthreads();
@@ -68,6 +71,23 @@ __global__ void __launch_bounds__(kMapThreads) rowmap_kernel(
     }
     if (tid == kMapThreads - 1) offsets[B] = part[tid];
     if (any_bad) atomicOr(status, ADWIN_DEV_WINDOW);
+    if (offsets_win) {   // the same scan over the effective windows
+      __syncthreads();
+      part[tid] = sum_win;
+      __syncthreads();
+      for (int o = 1; o < kMapThreads; o <<= 1) {
+        const int64_t v = (tid >= o) ? part[tid - o] : 0;
+        __syncthreads();
+        part[tid] += v;
+        __syncthreads();
+      }
+      int64_t run_win = part[tid] - sum_win;
+      for (int64_t b = b0; b < b1; ++b) {
+        offsets_win[b] = run_win;
+        run_win += ewin[b];
+      }
+      if (tid == kMapThreads - 1) offsets_win[B] = part[tid];
+    }
     return;
   }
   const int64_t n = B * T;
@@ -89,8 +109,9 @@ __global__ void __launch_bounds__(kMapThreads) rowmap_kernel(
 }
 
 cudaError_t launch_rowmap(const int32_t* window, const int32_t* rollout_len, int64_t B, int64_t T,
-                          int flags, void* workspace, float* kl, float* logratio, float* gsq,
-                          float* lse_s, float* lse_t, int32_t* status, cudaStream_t s) {
+                          int flags, void* workspace, bool with_window_offsets, float* kl,
+                          float* logratio, float* gsq, float* lse_s, float* lse_t, int32_t* status,
+                          cudaStream_t s) {
   const WorkspaceLayout w = workspace_layout(B);
   char* base = static_cast<char*>(workspace);
   const int64_t n = B * T;
@@ -99,6 +120,7 @@ cudaError_t launch_rowmap(const int32_t* window, const int32_t* rollout_len, int
   if (fill_blocks < 1) fill_blocks = 1;
   rowmap_kernel<<<(int)(1 + fill_blocks), kMapThreads, 0, s>>>(
       window, rollout_len, B, T, flags, reinterpret_cast<int64_t*>(base + w.off_offsets),
+      with_window_offsets ? reinterpret_cast<int64_t*>(base + w.off_offsets_win) : nullptr,
       reinterpret_cast<int32_t*>(base + w.off_range), reinterpret_cast<int32_t*>(base + w.off_ewin),
       kl, logratio, gsq, lse_s, lse_t, status);
   return cudaGetLastError();
