@@ -62,8 +62,8 @@ def measured_peak():
 
 # DRAM bytes per processed row of the staged kernel, from the committed ncu capture
 # (profiles/kl_staged_bf16_small_case_full.md), valid for the kernel source with this fingerprint.
-TRAFFIC_BYTES_PER_ROW = 856860
-TRAFFIC_KERNEL_SHA = "f589595c7073be11"
+TRAFFIC_BYTES_PER_ROW = 856940
+TRAFFIC_KERNEL_SHA = "63b30a9d15568918"
 
 
 def recorded_traffic(rows):
