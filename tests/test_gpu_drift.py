@@ -99,3 +99,30 @@ def test_drift_curves_over_many_rollouts_and_long_horizons():
         want = (np.maximum.accumulate(r, axis=1) <= k).mean(axis=0)
         np.testing.assert_allclose(cur.survival[j].cpu().numpy(), want, rtol=0, atol=1e-15)
     np.testing.assert_array_equal(cur.worst_rank.cpu().numpy(), np.maximum.accumulate(r, axis=1))
+
+
+def test_config3_full_size_drift_on_sampled_rows():
+    """The drift pass at the size the bench times it (B=16, T=2048, V=151936): entropy and rank
+    against the oracle on sampled rows, the curves against the same ranks on the host."""
+    batch = synth.make_batch(3, device=DEV)
+    B, T, V = batch.shape
+    ks = (1, 5, 20)
+    got = api.adwin_teacher_drift(batch.teacher, batch.tokens, batch.rollout_len)
+    cur = api.adwin_drift_curves(got.entropy, got.rank, batch.rollout_len, ks)
+    torch.cuda.synchronize()
+    api.raise_on_dev_status(got.dev_status)
+    rng = np.random.default_rng(8)
+    tok = batch.tokens.cpu().numpy()
+    for b in range(B):
+        for t in sorted({0, T - 1} | {int(x) for x in rng.integers(0, T, 2)}):
+            H, r = O.teacher_drift_row(batch.teacher[b, t].double().cpu().numpy(), int(tok[b, t]))
+            assert abs(float(got.entropy[b, t]) - H) <= 2e-3 * max(1.0, abs(H))
+            assert int(got.rank[b, t]) == r
+    ranks = got.rank.cpu().numpy().astype(np.int64)
+    R = batch.rollout_len.cpu().numpy()
+    np.testing.assert_array_equal(cur.worst_rank.cpu().numpy(), np.maximum.accumulate(ranks, axis=1))
+    for j, k in enumerate(ks):
+        np.testing.assert_array_equal(cur.survival[j].cpu().numpy(), O.topk_survival(ranks, R, k))
+    assert (cur.n_active.cpu().numpy() == B).all()
+    bf = np.exp(got.entropy.double().cpu().numpy()).mean(axis=0)
+    np.testing.assert_allclose(cur.bf_mean.cpu().numpy(), bf, rtol=1e-12)

@@ -122,3 +122,41 @@ def test_weighted_pass_with_the_costs_as_coefficients_is_the_sampled_mode():
                                               grad_dtype=torch.float32, flags=api.ZERO_TAIL)
     torch.cuda.synchronize()
     assert torch.equal(plain.grad, again.grad) and torch.equal(plain.gsq, again.gsq)
+
+
+def test_config3_full_size_two_pass_path_on_sampled_rows():
+    """The return-to-go path at the size the bench times it (B=16, T=2048, V=151936): the scan
+    against the oracle on every sequence, the weighted gradient on sampled rows."""
+    gamma, alpha = 0.9, 1.0
+    batch = synth.make_batch(3, device=DEV)
+    B, T, V = batch.shape
+    w, r = batch.window.cpu().numpy(), batch.rollout_len.cpu().numpy()
+    first = api.adwin_opd_kl_fwd_bwd(batch.student, batch.teacher, batch.tokens, batch.window,
+                                     batch.rollout_len)
+    rtg = api.adwin_return_to_go(first.logratio, batch.window, batch.rollout_len, gamma)
+    sentinel = 7.0
+    grad = torch.full((B, T, V), sentinel, dtype=torch.bfloat16, device=DEV)
+    got = api.adwin_opd_kl_fwd_bwd_weighted(batch.student, batch.teacher, batch.tokens,
+                                            batch.window, batch.rollout_len, rtg,
+                                            grad_scale=alpha, grad=grad)
+    torch.cuda.synchronize()
+    api.raise_on_dev_status(got.dev_status)
+    _check_rtg(rtg, first.logratio.double().cpu().numpy(), w, r, gamma, 0)
+    rng = np.random.default_rng(4)
+    coef = rtg.double().cpu().numpy()
+    tokens = batch.tokens.cpu().numpy()
+    rows, want, want_q = [], [], []
+    for b in range(B):
+        for t in sorted({0, int(w[b]) - 1} | {int(x) for x in rng.integers(0, int(w[b]), 2)}):
+            g, q = O.row_weighted(batch.student[b, t].double().cpu().numpy(), int(tokens[b, t]),
+                                  alpha, coef[b, t])
+            rows.append((b, t))
+            want.append(g)
+            want_q.append(q)
+    bs = torch.tensor([b for b, _ in rows], device=DEV)
+    ts = torch.tensor([t for _, t in rows], device=DEV)
+    P.check_grad_rows(grad[bs, ts].double().cpu().numpy(), np.stack(want), 2e-3, store=2.0 ** -8)
+    q = got.gsq[bs, ts].double().cpu().numpy()
+    assert (np.abs(q - np.array(want_q)) <= P.RTOL_GSQ * np.array(want_q) + 1e-30).all()
+    for b in range(B):
+        assert (grad[b, int(w[b]):] == sentinel).all()
