@@ -118,9 +118,12 @@ size_t adwin_workspace_bytes(int64_t B, int64_t T, int64_t V, int dtype, int fla
  * workspace    : >= adwin_workspace_bytes(...) bytes, 256-byte aligned; contents undefined after
  * dev_status   : one int32 the caller zeroed; bits are OR-ed in
  *
- * The staged (fast) kernel needs 16-byte aligned logits / gradient base pointers, row strides
- * that are multiples of 16 bytes and V*sizeof(element) a multiple of 16; any other layout runs
- * through the shape-agnostic kernel with identical results up to rounding order.
+ * Two kernels do the work, with identical results up to rounding order.  Rows whose gradient is
+ * written go to the staged cluster kernel (two sweeps with the row kept on chip), which needs
+ * 16-byte aligned logits / gradient base pointers, row strides that are multiples of 16 bytes and
+ * V*sizeof(element) a multiple of 16.  Rows without gradient (a call with grad_student == NULL,
+ * or the rows past the window of an ADWIN_RANGE_FULL call) and every other layout go to the
+ * streaming kernel, one CTA per row.  ADWIN_FORCE_GENERIC / ADWIN_FORCE_STAGED override the choice.
  */
 int adwin_opd_kl_fwd_bwd(const void* student_logits, const void* teacher_logits, int dtype,
                          int64_t B, int64_t T, int64_t V, int64_t ld, const int32_t* tokens,
