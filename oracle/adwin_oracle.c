@@ -17,8 +17,15 @@
  * E_{y~p}[c]=KL; gradients against central finite differences, zero row sum and the
  * expectation identity of Appendix A.1; window mask against brute-force prefix sums;
  * rho/SNR/L_next against closed forms, hand tables and a literal dot-product cosine.
- * The parameter-space cosine of Section 4.2 (gradients in R^d through the model Jacobian) is
- * NOT computed here: parity unpinned for that quantity (out of scope: it needs a model).
+ * The fused LM-head form (logits = hidden states times an output embedding; oracle functions in
+ * adwin_oracle.py, which call the per-row definition below on float64 logits) is pinned in
+ * tests/test_oracle_lmhead.py: explicit loops for the products, equality with this file's batch
+ * function on exactly representable logits, central differences with respect to hidden states and
+ * LM-head weight, nothing from positions outside the window, and the LM-head-weight-space cosine
+ * against its Gram form, the orthonormal case (= logit-space rho) and the shared-hidden-state case.
+ * The cosine of Section 4.2 over ALL model parameters (gradients in R^d through the whole model's
+ * Jacobian) is NOT computed here: parity unpinned for that quantity (out of scope: it needs a
+ * model); the LM-head weight is the one parameter block this path can see.
  *
  * No blocking, fusion or reordering: every function below is the definition written out.
  */
@@ -29,6 +36,7 @@
 
 #define ORACLE_F32 0
 #define ORACLE_BF16 1
+#define ORACLE_F64 2 /* logits that are already double (formed from hidden states and an LM head) */
 
 #define ORACLE_MODE_FULL_KL 0 /* gradient of the per-token reverse KL of Eq. 2 */
 #define ORACLE_MODE_SAMPLED 1 /* gamma = 0 score-function estimator, Eq. 4 */
@@ -43,6 +51,8 @@
 static double load_logit(const void *base, int dtype, int64_t idx) {
   if (dtype == ORACLE_F32) {
     return (double)((const float *)base)[idx];
+  } else if (dtype == ORACLE_F64) {
+    return ((const double *)base)[idx];
   } else {
     uint32_t bits = ((uint32_t)((const uint16_t *)base)[idx]) << 16;
     float f;

@@ -215,3 +215,128 @@ def topk_survival(rank, rollout_len, k: int):
     lib().adwin_oracle_topk_survival(_p(rank), _p(rollout_len), ctypes.c_int64(B),
                                      ctypes.c_int64(T), ctypes.c_int64(int(k)), _p(out))
     return out
+
+
+# --------------------------------------------------------------------------------------------
+# Fused LM-head form: the two policies of Eq. 2 are softmax(H W^T), hidden states times an output
+# embedding, and the quantities wanted are the same per-token scalars plus the gradients of the
+# windowed loss with respect to the student's hidden states and LM-head weight.  Written as the
+# definition: form the logits with a float64 matrix product (numpy's matmul is the library
+# primitive of this step), hand every processed row to the per-row definition above, then apply
+# the chain rule  dH_s = G W_s,  dW_s = G^T H_s  with G the window-masked logit gradient.
+# --------------------------------------------------------------------------------------------
+F64 = 2
+
+
+def widen(a):
+    """Stored values (float32 / float64, or uint16 bf16 bit patterns) exactly as float64."""
+    a = np.ascontiguousarray(a)
+    if a.dtype in (np.uint16, np.int16):
+        return (a.view(np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    if a.dtype in (np.float32, np.float64):
+        return a.astype(np.float64)
+    raise TypeError(f"expected float32/float64 or bf16 bits (uint16), got {a.dtype}")
+
+
+def _rows_f64_logits(z, u, tokens, window, rollout_len, grad_scale, grad_mode, flags):
+    """Per-row definition on float64 logits z, u [B,T,V]; gradient zero outside the window."""
+    B, T, V = z.shape
+    kl = np.empty((B, T)); c = np.empty((B, T)); gsq = np.empty((B, T))
+    ls = np.empty((B, T)); lt = np.empty((B, T))
+    grad = np.zeros((B, T, V), dtype=np.float64)
+    rc = lib().adwin_oracle_opd_kl_fwd_bwd(
+        _p(z), _p(u), ctypes.c_int(F64), ctypes.c_int64(B), ctypes.c_int64(T), ctypes.c_int64(V),
+        ctypes.c_int64(V), _p(tokens), _p(window), _p(rollout_len), ctypes.c_double(grad_scale),
+        ctypes.c_int(grad_mode), ctypes.c_int(flags), _p(grad), ctypes.c_int64(V), _p(kl), _p(c),
+        _p(gsq), _p(ls), _p(lt))
+    if rc != 0:
+        raise ValueError(f"oracle rejected window / rollout lengths (code {rc})")
+    return kl, c, gsq, ls, lt, grad
+
+
+def lmhead_logits(H, W):
+    """z[b,t,k] = sum_j H[b,t,j] W[k,j] in float64 (stored values widened exactly)."""
+    return widen(H) @ widen(W).T
+
+
+def lmhead_fwd_bwd(Hs, Ws, Ht, Wt, tokens, window, rollout_len=None, grad_scale: float = 1.0,
+                   grad_mode: int = MODE_FULL_KL, flags: int = 0):
+    """The OPD divergence of Eq. 2 with both policies given as hidden states times an LM head.
+
+    Hs [B,T,d_s], Ws [V,d_s] (student), Ht [B,T,d_t], Wt [V,d_t] (teacher); tokens, window,
+    rollout_len, grad_scale, grad_mode as in opd_kl_fwd_bwd; flags: FLAG_RANGE_FULL only.
+    One sequence at a time:
+      z = Hs[b] Ws^T, u = Ht[b] Wt^T                       (the logits of Eq. 2's two policies)
+      kl, logratio, gsq, lse per processed position        (the per-row definition)
+      G[b,t,:] = d loss / d z[b,t,:] for t inside the window, zero elsewhere
+      dH[b,t,:] = G[b,t,:] Ws                              chain rule through z = H_s W_s^T
+      dW       += G[b]^T Hs[b]
+    Returns dict(kl, logratio, gsq, lse_s, lse_t [B,T]; dH [B,T,d_s]; dW [V,d_s]), float64.
+    """
+    Hs64, Ws64, Ht64, Wt64 = widen(Hs), widen(Ws), widen(Ht), widen(Wt)
+    B, T, ds = Hs64.shape
+    V = Ws64.shape[0]
+    assert Ws64.shape == (V, ds) and Ht64.shape[:2] == (B, T) and Wt64.shape == (V, Ht64.shape[2])
+    tokens = _i32(tokens).reshape(B, T)
+    window = _i32(window)
+    rollout_len = _i32(rollout_len) if rollout_len is not None else np.full(B, T, np.int32)
+    out = {k: np.zeros((B, T)) for k in ("kl", "logratio", "gsq", "lse_s", "lse_t")}
+    dH = np.zeros((B, T, ds))
+    dW = np.zeros((V, ds))
+    for b in range(B):
+        z = (Hs64[b] @ Ws64.T)[None]
+        u = (Ht64[b] @ Wt64.T)[None]
+        kl, c, gsq, ls, lt, G = _rows_f64_logits(z, u, tokens[b:b + 1], window[b:b + 1],
+                                                 rollout_len[b:b + 1], grad_scale, grad_mode,
+                                                 flags & FLAG_RANGE_FULL)
+        for name, val in (("kl", kl), ("logratio", c), ("gsq", gsq), ("lse_s", ls), ("lse_t", lt)):
+            out[name][b] = val[0]
+        dH[b] = G[0] @ Ws64
+        dW += G[0].T @ Hs64[b]
+    out["dH"] = dH
+    out["dW"] = dW
+    return out
+
+
+def lmhead_weight_cosine(Hs, Ws, Ht, Wt, tokens, rollout_len, candidates, grad_scale: float = 1.0,
+                         grad_mode: int = MODE_FULL_KL):
+    """Prefix-versus-full cosine of Section 4.2 in the space of the student's LM-head weight.
+
+    For every candidate length L the prefix gradient is dW^(L) = sum over sequences and positions
+    t < min(L, R_b) of g[b,t] h[b,t]^T, the full-horizon probe reference dW^full the same sum over
+    t < R_b.  Literally: build both matrices, take <A,B> / (|A| |B|).  Returns
+    dict(micro [K] = cosine after summing over the batch, macro [K] = mean over sequences of the
+    per-sequence cosine, per_seq [B,K]).  A zero full norm gives cosine 1, a zero prefix norm 0.
+    """
+    Hs64, Ws64, Ht64, Wt64 = widen(Hs), widen(Ws), widen(Ht), widen(Wt)
+    B, T, ds = Hs64.shape
+    V = Ws64.shape[0]
+    tokens = _i32(tokens).reshape(B, T)
+    rollout_len = _i32(rollout_len) if rollout_len is not None else np.full(B, T, np.int32)
+    cands = [int(L) for L in np.asarray(candidates).ravel()]
+
+    def cos(a, b):
+        na, nb = np.sqrt(np.sum(a * a)), np.sqrt(np.sum(b * b))
+        if not nb > 0:
+            return 1.0
+        return float(np.sum(a * b) / (na * nb)) if na > 0 else 0.0
+
+    full_b = np.zeros((B, V, ds))
+    pre_b = np.zeros((len(cands), B, V, ds))
+    for b in range(B):
+        z = (Hs64[b] @ Ws64.T)[None]
+        u = (Ht64[b] @ Wt64.T)[None]
+        G = _rows_f64_logits(z, u, tokens[b:b + 1], rollout_len[b:b + 1], rollout_len[b:b + 1],
+                             grad_scale, grad_mode, 0)[5][0]
+        for t in range(T):
+            if t < rollout_len[b]:
+                outer = np.outer(G[t], Hs64[b, t])
+                full_b[b] += outer
+                for j, L in enumerate(cands):
+                    if t < L:
+                        pre_b[j, b] += outer
+    per_seq = np.array([[cos(pre_b[j, b], full_b[b]) for j in range(len(cands))]
+                        for b in range(B)]).reshape(B, len(cands))
+    micro = np.array([cos(pre_b[j].sum(axis=0), full_b.sum(axis=0)) for j in range(len(cands))])
+    return dict(micro=micro, macro=per_seq.mean(axis=0) if B else np.ones(len(cands)),
+                per_seq=per_seq)
