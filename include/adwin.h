@@ -48,7 +48,9 @@ typedef enum {
   ADWIN_DEV_NONFINITE = 2,   /* a processed row produced a non-finite log-sum-exp */
   ADWIN_DEV_TIMEOUT = 4,     /* a bounded on-chip wait ran out; outputs of this call are invalid */
   ADWIN_DEV_BOUNDS = 8,      /* an internal index check failed; outputs of this call are invalid */
-  ADWIN_DEV_WINDOW = 16      /* some W_b < 0, R_b < 0 or R_b > T; the value was clamped to [0,T] */
+  ADWIN_DEV_WINDOW = 16,     /* some W_b < 0, R_b < 0 or R_b > T; the value was clamped to [0,T] */
+  ADWIN_DEV_WORKSPACE = 32   /* more processed positions than the workspace was sized for (the
+                                max_rows bound of the fused LM-head call); nothing was computed */
 } adwin_dev_status_t;
 
 typedef enum { ADWIN_F32 = 0, ADWIN_BF16 = 1 } adwin_dtype_t;
@@ -233,6 +235,49 @@ int adwin_teacher_drift(const void* teacher_logits, int dtype, int64_t B, int64_
 int adwin_drift_curves(const float* entropy, const int32_t* rank, const int32_t* rollout_len,
                        int64_t B, int64_t T, const int32_t* ks, int32_t K, int32_t* worst_rank,
                        double* survival, double* bf_mean, int32_t* n_active, void* cuda_stream);
+
+/*
+ * The same divergence with both policies given as hidden states times an output embedding (the
+ * form Eq. 2's policies have in a language model: pi = softmax(h W^T)), fused so that the logits
+ * are never written to memory:
+ *     z[b,t,:] = hidden_student[b,t,:] W_s^T,      u[b,t,:] = hidden_teacher[b,t,:] W_t^T,
+ * then kl, logratio, gsq, lse_student, lse_teacher exactly as adwin_opd_kl_fwd_bwd defines them on
+ * (z, u), and the gradients of the windowed loss with respect to the student's hidden states and
+ * output embedding,
+ *     grad_hidden[b,t,:] = G[b,t,:] W_s   for t < E_b,        grad_w = sum_{b, t < E_b} G[b,t,:]^T h_s[b,t,:],
+ * where G is the logit gradient of the selected estimator (adwin_grad_mode_t, alpha = grad_scale).
+ * grad_w is the student's LM-head block of the parameter-space gradient that Section 4.2's cosine
+ * is defined on.  The products run on the tensor cores in bf16 with fp32 accumulation; G is
+ * rounded to bf16 once before the two gradient products.
+ *
+ * hidden_student [B,T,d_s], w_student [V,d_s], hidden_teacher [B,T,d_t], w_teacher [V,d_t]:
+ *                bf16, contiguous, 16-byte aligned; V, d_s, d_t multiples of 8
+ * tokens, window, rollout_len, grad_scale, grad_mode: as in adwin_opd_kl_fwd_bwd
+ * flags        : ADWIN_RANGE_FULL (per-token scalars for every t < R_b; gradients still from
+ *                t < E_b only) and ADWIN_ZERO_TAIL (zero-fill grad_hidden rows t >= E_b; they are
+ *                left untouched otherwise)
+ * grad_hidden  : [B,T,d_s] of grad_hidden_dtype (ADWIN_F32 / ADWIN_BF16), or NULL
+ * grad_w       : [V,d_s] fp32, overwritten (not accumulated into), or NULL
+ * kl, logratio : [B,T] fp32, required.   gsq, lse_student, lse_teacher: [B,T] fp32 or NULL
+ * max_rows     : an upper bound on the number of processed positions, sum_b E_b (sum_b R_b with
+ *                ADWIN_RANGE_FULL), which sizes the workspace; <= 0 means B*T.  If the lengths on
+ *                the device exceed it, ADWIN_DEV_WORKSPACE is raised and nothing is computed.
+ * workspace    : >= adwin_lmhead_workspace_bytes(...) bytes, 1024-byte aligned; it holds compact
+ *                copies of the processed hidden states, partial row statistics and, when a
+ *                gradient is requested, G in bf16 (2 V bytes per processed position)
+ * Errors as in adwin_opd_kl_fwd_bwd; shapes this path cannot take return ADWIN_ERR_UNSUPPORTED.
+ */
+size_t adwin_lmhead_workspace_bytes(int64_t B, int64_t T, int64_t V, int64_t d_s, int64_t d_t,
+                                    int64_t max_rows, int flags, int with_grad);
+int adwin_opd_kl_lmhead_fwd_bwd(const void* hidden_student, const void* w_student,
+                                const void* hidden_teacher, const void* w_teacher, int64_t B,
+                                int64_t T, int64_t V, int64_t d_s, int64_t d_t,
+                                const int32_t* tokens, const int32_t* window,
+                                const int32_t* rollout_len, float grad_scale, int grad_mode,
+                                int flags, void* grad_hidden, int grad_hidden_dtype, float* grad_w,
+                                float* kl, float* logratio, float* gsq, float* lse_student,
+                                float* lse_teacher, int64_t max_rows, void* workspace,
+                                size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
 
 /*
  * The same pass for logits that live in HOST memory (pinned memory gives asynchronous copies).

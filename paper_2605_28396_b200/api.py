@@ -19,7 +19,7 @@ OK = 0
 F32, BF16 = 0, 1
 GRAD_FULL_KL, GRAD_SAMPLED = 0, 1
 ZERO_TAIL, RANGE_FULL, FORCE_GENERIC, FORCE_STAGED = 1, 2, 4, 8
-DEV_TOKEN_RANGE, DEV_NONFINITE, DEV_TIMEOUT, DEV_BOUNDS, DEV_WINDOW = 1, 2, 4, 8, 16
+DEV_TOKEN_RANGE, DEV_NONFINITE, DEV_TIMEOUT, DEV_BOUNDS, DEV_WINDOW, DEV_WORKSPACE = 1, 2, 4, 8, 16, 32
 ALIGN_DEGENERATE, ALIGN_NONE_ADMISSIBLE = 1, 2
 DEFAULT_CANDIDATES = (64, 128, 256, 512, 1024, 2048)   # Section 5.1, Training Details
 RHO_STAR = math.sqrt(2.0) / 2.0                          # Section 4.2, threshold equation
@@ -29,7 +29,7 @@ EXPORTS = ("adwin_version", "adwin_status_string", "adwin_workspace_bytes",
            "adwin_host_staging_bytes", "adwin_opd_kl_fwd_bwd_host",
            "adwin_no_alloc_max_sequences", "adwin_opd_kl_fwd_bwd_no_alloc",
            "adwin_return_to_go", "adwin_opd_kl_fwd_bwd_weighted", "adwin_teacher_drift",
-           "adwin_drift_curves")
+           "adwin_drift_curves", "adwin_lmhead_workspace_bytes", "adwin_opd_kl_lmhead_fwd_bwd")
 
 _lib = None
 
@@ -88,6 +88,14 @@ def lib():
                                           vp]
         L.adwin_drift_curves.restype = ctypes.c_int
         L.adwin_drift_curves.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, vp, vp, vp, vp]
+        L.adwin_lmhead_workspace_bytes.restype = sz
+        L.adwin_lmhead_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, i64, ctypes.c_int,
+                                                   ctypes.c_int]
+        L.adwin_opd_kl_lmhead_fwd_bwd.restype = ctypes.c_int
+        L.adwin_opd_kl_lmhead_fwd_bwd.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, i64, vp, vp,
+                                                  vp, f32, ctypes.c_int, ctypes.c_int, vp,
+                                                  ctypes.c_int, vp, vp, vp, vp, vp, vp, i64, vp,
+                                                  sz, vp, vp]
         _lib = L
     return _lib
 
@@ -205,7 +213,8 @@ def raise_on_dev_status(dev_status, allow=0):
     """Synchronising read of the device status word; raises on bits outside ``allow``."""
     bits = int(dev_status.item())
     if bits & ~allow:
-        names = {1: "TOKEN_RANGE", 2: "NONFINITE", 4: "TIMEOUT", 8: "BOUNDS", 16: "WINDOW"}
+        names = {1: "TOKEN_RANGE", 2: "NONFINITE", 4: "TIMEOUT", 8: "BOUNDS", 16: "WINDOW",
+                 32: "WORKSPACE"}
         raise RuntimeError("adwin device status: " +
                            "|".join(n for b, n in names.items() if bits & b))
     return bits
@@ -347,3 +356,59 @@ def adwin_drift_curves(entropy, rank, rollout_len=None, ks=(1, 5, 20)):
                                     _ptr(ks_t), K, _ptr(o.worst_rank), _ptr(o.survival),
                                     _ptr(o.bf_mean), _ptr(o.n_active), _stream(dev)))
     return o
+
+
+def adwin_lmhead_workspace_bytes(B, T, V, d_s, d_t, max_rows=0, flags=0, with_grad=True) -> int:
+    return int(lib().adwin_lmhead_workspace_bytes(B, T, V, d_s, d_t, int(max_rows), int(flags),
+                                                  1 if with_grad else 0))
+
+
+def adwin_opd_kl_lmhead_fwd_bwd(hidden_student, w_student, hidden_teacher, w_teacher, tokens,
+                                window, rollout_len=None, *, grad_scale=1.0,
+                                grad_mode=GRAD_FULL_KL, flags=0, grad_hidden=None, grad_w=None,
+                                want_gsq=True, want_lse=False, max_rows=0, workspace=None,
+                                dev_status=None):
+    """Fused LM-head form: policies given as hidden states times output embeddings (adwin.h).
+
+    hidden_* [B,T,d] and w_* [V,d] bf16 contiguous device tensors.  grad_hidden ([B,T,d_s], bf16 or
+    fp32) and grad_w ([V,d_s] fp32) are caller-allocated and optional.  Returns a namespace with
+    kl, logratio, gsq, lse_s, lse_t, dev_status, workspace.
+    """
+    B, T, ds = hidden_student.shape
+    V = w_student.shape[0]
+    dt = hidden_teacher.shape[2]
+    dev = hidden_student.device
+    for t in (hidden_student, w_student, hidden_teacher, w_teacher):
+        if t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise TypeError("hidden states and LM heads must be contiguous bf16 tensors")
+    if w_student.shape != (V, ds) or hidden_teacher.shape[:2] != (B, T) or \
+            w_teacher.shape != (V, dt):
+        raise ValueError("shape mismatch")
+    for g in (grad_hidden, grad_w):
+        if g is not None and not g.is_contiguous():
+            raise ValueError("gradient tensors must be contiguous")
+    kl = torch.empty((B, T), dtype=torch.float32, device=dev)
+    logratio = torch.empty((B, T), dtype=torch.float32, device=dev)
+    gsq = torch.empty((B, T), dtype=torch.float32, device=dev) if want_gsq else None
+    lse_s = torch.empty((B, T), dtype=torch.float32, device=dev) if want_lse else None
+    lse_t = torch.empty((B, T), dtype=torch.float32, device=dev) if want_lse else None
+    with_grad = grad_hidden is not None or grad_w is not None
+    need = adwin_lmhead_workspace_bytes(B, T, V, ds, dt, max_rows, flags, with_grad)
+    if workspace is None:
+        workspace = torch.empty(need + 1024, dtype=torch.uint8, device=dev)
+    off = (-workspace.data_ptr()) % 1024
+    ws_ptr = ctypes.c_void_p(workspace.data_ptr() + off)
+    ws_bytes = workspace.numel() - off
+    if dev_status is None:
+        dev_status = torch.zeros(1, dtype=torch.int32, device=dev)
+    gh_dtype = _dtype_code(grad_hidden.dtype) if grad_hidden is not None else F32
+    if grad_w is not None and grad_w.dtype != torch.float32:
+        raise TypeError("grad_w must be float32")
+    _check(lib().adwin_opd_kl_lmhead_fwd_bwd(
+        _ptr(hidden_student), _ptr(w_student), _ptr(hidden_teacher), _ptr(w_teacher), B, T, V, ds,
+        dt, _ptr(tokens), _ptr(window), _ptr(rollout_len), float(grad_scale), int(grad_mode),
+        int(flags), _ptr(grad_hidden), gh_dtype, _ptr(grad_w), _ptr(kl), _ptr(logratio),
+        _ptr(gsq), _ptr(lse_s), _ptr(lse_t), int(max_rows), ws_ptr, ws_bytes, _ptr(dev_status),
+        _stream(dev)))
+    return SimpleNamespace(kl=kl, logratio=logratio, gsq=gsq, lse_s=lse_s, lse_t=lse_t,
+                           dev_status=dev_status, workspace=workspace)

@@ -313,4 +313,74 @@ int adwin_probe_align(const float* kl, const float* logratio, const float* gsq,
   return ADWIN_OK;
 }
 
+size_t adwin_lmhead_workspace_bytes(int64_t B, int64_t T, int64_t V, int64_t d_s, int64_t d_t,
+                                    int64_t max_rows, int flags, int with_grad) {
+  if (B < 0) B = 0;
+  if (T < 0) T = 0;
+  if (V < 1) V = 1;
+  if (d_s < 1) d_s = 1;
+  if (d_t < 1) d_t = 1;
+  return lmhead_workspace_bytes(B, T, V, d_s, d_t, max_rows, with_grad != 0,
+                                (flags & ADWIN_RANGE_FULL) != 0);
+}
+
+int adwin_opd_kl_lmhead_fwd_bwd(const void* hidden_student, const void* w_student,
+                                const void* hidden_teacher, const void* w_teacher, int64_t B,
+                                int64_t T, int64_t V, int64_t d_s, int64_t d_t,
+                                const int32_t* tokens, const int32_t* window,
+                                const int32_t* rollout_len, float grad_scale, int grad_mode,
+                                int flags, void* grad_hidden, int grad_hidden_dtype, float* grad_w,
+                                float* kl, float* logratio, float* gsq, float* lse_student,
+                                float* lse_teacher, int64_t max_rows, void* workspace,
+                                size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+  if (grad_mode != ADWIN_GRAD_FULL_KL && grad_mode != ADWIN_GRAD_SAMPLED) return ADWIN_ERR_DTYPE;
+  if (flags & ~(ADWIN_RANGE_FULL | ADWIN_ZERO_TAIL)) return ADWIN_ERR_DTYPE;
+  if (grad_hidden && grad_hidden_dtype != ADWIN_F32 && grad_hidden_dtype != ADWIN_BF16)
+    return ADWIN_ERR_DTYPE;
+  if (B < 0 || T < 0 || B > 65536 || T > kMaxT || V < 1 || V > kMaxV || d_s < 1 || d_t < 1 ||
+      d_s > (int64_t(1) << 20) || d_t > (int64_t(1) << 20))
+    return ADWIN_ERR_SHAPE;
+  if (!dev_status) return ADWIN_ERR_NULL;
+  if (B == 0 || T == 0) return ADWIN_OK;
+  if (!hidden_student || !w_student || !hidden_teacher || !w_teacher || !tokens || !window ||
+      !kl || !logratio)
+    return ADWIN_ERR_NULL;
+  if ((V % 8) || (d_s % 8) || (d_t % 8) || B * T > (int64_t(1) << 30)) return ADWIN_ERR_UNSUPPORTED;
+  if (!aligned(hidden_student, 16) || !aligned(w_student, 16) || !aligned(hidden_teacher, 16) ||
+      !aligned(w_teacher, 16) || !aligned(grad_hidden, 16) || !aligned(grad_w, 16) ||
+      !aligned(tokens, 4) || !aligned(window, 4) || !aligned(rollout_len, 4) || !aligned(kl, 4) ||
+      !aligned(logratio, 4) || !aligned(gsq, 4) || !aligned(lse_student, 4) ||
+      !aligned(lse_teacher, 4) || !aligned(dev_status, 4))
+    return ADWIN_ERR_ALIGN;
+  const bool want_grad = grad_hidden || grad_w;
+  if (!workspace || !aligned(workspace, 1024) ||
+      workspace_bytes < lmhead_workspace_bytes(B, T, V, d_s, d_t, max_rows, want_grad,
+                                               (flags & ADWIN_RANGE_FULL) != 0))
+    return ADWIN_ERR_WORKSPACE;
+  const int sms = sm_count_of_current_device();
+  if (sms <= 0) return ADWIN_ERR_CUDA;
+  if (launch_lmhead(hidden_student, w_student, hidden_teacher, w_teacher, B, T, V, d_s, d_t, tokens,
+                    window, rollout_len, grad_scale, grad_mode, flags, grad_hidden,
+                    grad_hidden_dtype, grad_w, kl, logratio, gsq, lse_student, lse_teacher,
+                    workspace, max_rows, dev_status, sms,
+                    static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return ADWIN_ERR_CUDA;
+  return ADWIN_OK;
+}
+
+#ifdef ADWIN_DEV_EXPORTS
+// Development build only: the tensor-core GEMM on its own, C = A B (bf16 in, fp32 or bf16 out).
+int adwin_dev_gemm(const void* A, int64_t lda, int a_mn, const void* Bm, int64_t ldb, int b_mn,
+                   int64_t M, int64_t N, int64_t K, void* C, int64_t ldc, int c_bf16,
+                   int32_t* dev_status, void* cuda_stream) {
+  const int sms = sm_count_of_current_device();
+  if (sms <= 0) return ADWIN_ERR_CUDA;
+  return launch_tc_gemm(A, lda, a_mn != 0, Bm, ldb, b_mn != 0, M, N, K, C, ldc, c_bf16 != 0,
+                        nullptr, nullptr, nullptr, dev_status, sms,
+                        static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+             ? ADWIN_OK
+             : ADWIN_ERR_CUDA;
+}
+#endif
+
 }  // extern "C"
