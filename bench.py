@@ -47,6 +47,12 @@ def parse():
     ap.add_argument("--seqs", type=int, default=None, help="override B (profiling a small case only)")
     ap.add_argument("--positions", type=int, default=None,
                     help="override T (profiling a small case only)")
+    ap.add_argument("--no-side", action="store_true",
+                    help="skip the side measurements (profiling a small case only)")
+    ap.add_argument("--lmhead-seqs", type=int, default=None,
+                    help="override B of the fused LM-head side measurement (profiling only)")
+    ap.add_argument("--lmhead-positions", type=int, default=None,
+                    help="override T of the fused LM-head side measurement (profiling only)")
     return ap.parse_args()
 
 
@@ -60,22 +66,36 @@ def measured_peak():
     return 6650.0, "fallback 6.65 TB/s (of fallback)"
 
 
-# DRAM bytes per processed row of the staged kernel, from the committed ncu capture
-# (profiles/kl_staged_bf16_small_case_full.md), valid for the kernel source with this fingerprint.
-TRAFFIC_BYTES_PER_ROW = 856940
+# DRAM bytes READ per processed row of the staged kernel, from the committed ncu capture of a
+# small case (960 rows), valid for the kernel source with this fingerprint.  The capture's write
+# counter is not scaled: the last ~56 MB of a launch's gradient are still in L2 when the kernel
+# ends, a residue bounded by the L2 size that does not grow with the rows, so at full size the
+# writes are taken as the gradient bytes themselves.
+TRAFFIC_READ_BYTES_PER_ROW = 611598
 TRAFFIC_KERNEL_SHA = "63b30a9d15568918"
 
 
-def recorded_traffic(rows):
-    """DRAM bytes of one launch, scaled from the captured case by rows; None once the kernel source
-    has changed since the counters were taken."""
+def recorded_traffic(rows, V):
+    """DRAM bytes of one launch: the captured reads scaled by rows plus the gradient bytes written;
+    None once the kernel source has changed since the counters were taken."""
     import hashlib
     h = hashlib.sha256()
     for f in ("kl_staged.cu", "adwin_common.cuh"):
         h.update((ROOT / "paper_2605_28396_b200" / "csrc" / f).read_bytes())
     if h.hexdigest()[:16] != TRAFFIC_KERNEL_SHA:
         return None
-    return TRAFFIC_BYTES_PER_ROW * rows
+    return TRAFFIC_READ_BYTES_PER_ROW * rows + rows * V * 2
+
+
+def measured_tensor_peaks():
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        try:
+            d = json.loads(f.read_text())
+            return float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "MEASURED_PEAKS.json (of measured)"
+        except Exception:
+            pass
+    return 1590.0, 1400.0, "fallback 1.59 / 1.4 PFLOP/s (of fallback)"
 
 
 class ClockSampler:
@@ -307,8 +327,64 @@ def run_ours(args):
 
     # ---- the two-pass update with return-to-go weights (Eq. 3, gamma > 0), same batch: a read-only
     # pass for the costs, the scan over [B,T], the sampled-token gradient pass with the weights
+    side = rank == 0 and world == 1 and not args.no_side
+
+    def time_loop(fn, n, warm=3):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        if int(status.item()):
+            raise SystemExit("device status set by a side measurement")
+        return a.elapsed_time(b) / n
+
+    # ---- the same step back to back for >= 2 s with the clocks sampled: what the kernel does once
+    # the SM clock has settled under sustained load (nothing is set, only read)
+    sustained = None
+    if side:
+        n_sus = max(50, int(2200.0 / max(ms_step, 1e-3)))
+        sus_sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
+        sus_sampler.start()
+        time.sleep(0.2)
+        sus_ms = time_loop(step, n_sus, warm=0)
+        sus_clk = sus_sampler.stop()
+        mhz = sus_clk.get("sm_mhz")
+        sustained = {"steps": n_sus, "ms_per_step": sus_ms, "seconds": sus_ms * n_sus / 1e3,
+                     "tokens_per_s": rows / (sus_ms / 1e3), "sm_mhz_median": mhz,
+                     "ms_times_mhz": (sus_ms * mhz) if mhz else None,
+                     "achieved_gbs": rows * V * 6 / (sus_ms * 1e-3) / 1e9,
+                     "clocks": sus_clk}
+
+    # ---- scalars for every t < R_b and the gradient inside the window, one call (default dispatch:
+    # the staged kernel over the window rows, the streaming kernel over the rest of every rollout)
+    n2_line = None
+    if side:
+        ws2 = torch.empty(api.adwin_workspace_bytes(B, T, V), dtype=torch.uint8, device=dev)
+        n2out = None
+
+        def n2_step():
+            nonlocal n2out
+            n2out = api.adwin_opd_kl_fwd_bwd(batch.student, batch.teacher, batch.tokens,
+                                             batch.window, batch.rollout_len, grad=grad, out=n2out,
+                                             flags=api.RANGE_FULL, workspace=ws2, dev_status=status)
+        n2ms = time_loop(n2_step, 5)
+        allrows = int(batch.rollout_len.sum())
+        n2bytes = rows * V * 6 + (allrows - rows) * V * 4
+        peak_n2, _ = measured_peak()
+        n2_line = {"ms_per_step": n2ms, "positions": allrows, "rows_with_gradient": rows,
+                   "algorithmic_bytes": n2bytes, "achieved_gbs": n2bytes / (n2ms * 1e-3) / 1e9,
+                   "frac_of_measured_peak": n2bytes / (n2ms * 1e-3) / 1e9 / peak_n2,
+                   "launches_per_step": 3, "steps": 5,
+                   "path": "adwin_opd_kl_fwd_bwd (RANGE_FULL with gradient: rowmap, "
+                           "kl_staged_kernel over t < E_b, kl_generic_kernel over E_b <= t < R_b)"}
+
     rtg_line = None
-    if rank == 0 and world == 1:
+    if side:
         gamma, n_rtg = 0.9, 5
         probe = rtg = wout = None
 
@@ -345,7 +421,7 @@ def run_ours(args):
     # ---- the delayed full-rollout probe (Section 4.2) on the same batch: every position t < R_b,
     # read-only, followed by the audit; this is the pass that config 4 runs at T = 8192
     probe_line = None
-    if rank == 0 and world == 1:
+    if side:
         n_probe = 5
         pout = None
 
@@ -381,7 +457,7 @@ def run_ours(args):
     # ---- teacher-drift diagnostics (Section 3.1) over every position of the same batch: one read
     # of the teacher logits, then the survival / branching-factor curves
     drift_line = None
-    if rank == 0 and world == 1:
+    if side:
         n_drift = 5
         ks = torch.tensor([1, 5, 20], dtype=torch.int32, device=dev)
 
@@ -409,6 +485,80 @@ def run_ours(args):
                       "path": "adwin_teacher_drift -> adwin_drift_curves (timed together)"}
         if int(status.item()):
             raise SystemExit("device status set by the teacher-drift path")
+
+    # ---- config 4: the delayed full-rollout probe at its own shape (B=8, T=8192), read-only pass
+    # over every position followed by the audit
+    cfg4_line = None
+    if side and args.seqs is None and args.positions is None:
+        b4 = synth.make_batch(4, device=dev)
+        B4, T4, _ = b4.shape
+        ws4 = torch.empty(api.adwin_workspace_bytes(B4, T4, V), dtype=torch.uint8, device=dev)
+        o4 = None
+
+        def cfg4_step():
+            nonlocal o4
+            o4 = api.adwin_opd_kl_fwd_bwd(b4.student, b4.teacher, b4.tokens, b4.window,
+                                          b4.rollout_len, out=o4, flags=api.RANGE_FULL,
+                                          workspace=ws4, dev_status=status)
+            return api.adwin_probe_align(o4.kl, o4.logratio, o4.gsq, b4.window, b4.rollout_len)
+        c4ms = time_loop(cfg4_step, 5)
+        c4rows = int(b4.rollout_len.sum())
+        c4bytes = c4rows * V * 4
+        peak_4, _ = measured_peak()
+        cfg4_line = {"workload": "config4: B=8 T=8192 V=151936 bf16, W_b ~ U{512..4096}, R_b = T",
+                     "ms_per_step": c4ms, "positions": c4rows,
+                     "tokens_per_s": c4rows / (c4ms / 1e3), "algorithmic_bytes": c4bytes,
+                     "achieved_gbs": c4bytes / (c4ms * 1e-3) / 1e9,
+                     "frac_of_measured_peak": c4bytes / (c4ms * 1e-3) / 1e9 / peak_4,
+                     "launches_per_step": 2 + 3, "steps": 5,
+                     "path": "adwin_opd_kl_fwd_bwd (RANGE_FULL, no gradient: kl_generic_kernel) "
+                             "-> adwin_probe_align (timed together)"}
+        del b4, ws4, o4
+        torch.cuda.empty_cache()
+
+    # ---- config 5: the fused LM-head variant (hidden states x output embeddings, logits never
+    # materialised), forward statistics + gradients with respect to H_s and W_s; tensor roofline
+    lm_line = None
+    if side:
+        lb = synth.make_lmhead_batch(dev, B=args.lmhead_seqs, T=args.lmhead_positions)
+        LB, LT, ds = lb.hidden_student.shape
+        dt = lb.hidden_teacher.shape[2]
+        nw = int(torch.minimum(lb.window, lb.rollout_len).sum())
+        dH = torch.empty((LB, LT, ds), dtype=torch.bfloat16, device=dev)
+        dW = torch.empty((V, ds), dtype=torch.float32, device=dev)
+        lws = torch.empty(api.adwin_lmhead_workspace_bytes(LB, LT, V, ds, dt, nw, 0, True) + 1024,
+                          dtype=torch.uint8, device=dev)
+
+        def lm_step(with_grad=True):
+            return api.adwin_opd_kl_lmhead_fwd_bwd(
+                lb.hidden_student, lb.w_student, lb.hidden_teacher, lb.w_teacher, lb.tokens,
+                lb.window, lb.rollout_len, grad_hidden=dH if with_grad else None,
+                grad_w=dW if with_grad else None, max_rows=nw, workspace=lws, dev_status=status)
+        lm_ms = time_loop(lm_step, 5)
+        lm_fwd_ms = time_loop(lambda: lm_step(False), 5)
+        fl_fwd = 2.0 * nw * V * (ds + dt)
+        fl_all = 2.0 * fl_fwd + 2.0 * 2.0 * nw * V * ds
+        burst, sust, tsrc = measured_tensor_peaks()
+        ach = fl_all / (lm_ms * 1e-3) / 1e12
+        lm_line = {"workload": f"config5: B={LB} T={LT} V={V} H_s [B*T,{ds}] H_t [B*T,{dt}] bf16 "
+                               f"N(0,1), W_s, W_t bf16 N(0,0.02), W_b ~ U{{{max(1, LT // 16)}..{LT}}}, "
+                               "FULL_KL, dH_s bf16, dW_s fp32",
+                   "in_window_rows": nw, "ms_per_step": lm_ms, "tokens_per_s": nw / (lm_ms / 1e3),
+                   "forward_only_ms": lm_fwd_ms,
+                   "forward_only_tflops": fl_fwd / (lm_fwd_ms * 1e-3) / 1e12,
+                   "method_flops": fl_all, "steps": 5,
+                   "roofline": {"bound": "tensor", "achieved": ach, "peak": sust,
+                                "unit": "TFLOP/s", "frac": ach / sust, "traffic": None,
+                                "peak_burst": burst, "frac_of_burst": ach / burst,
+                                "peak_source": tsrc + ": sustained figure (a 100+ ms step under "
+                                               "the power cap); burst beside it",
+                                "flops": "in-window rows only: 2 N V (d_s+d_t) for each of the two "
+                                         "sweeps + 2 N V d_s each for dH_s and dW_s"},
+                   "launches_per_step": 9,
+                   "path": "adwin_opd_kl_lmhead_fwd_bwd: rowmap, plan, 2 gathers, lm_sweep "
+                           "(statistics), merge, lm_sweep (gradient), tc_gemm (dH_s), tc_gemm (dW_s)"}
+        del lb, dH, dW, lws
+        torch.cuda.empty_cache()
 
     # ---- end to end through the host-buffer entry point (copies inside the timed region)
     e2e = None
@@ -463,7 +613,7 @@ def run_ours(args):
     peak, peak_src = measured_peak()
     alg_bytes = rows * V * 6            # per launch on one GPU: 2 reads + 1 write of bf16 per entry
     achieved = alg_bytes / (kernel_ms * 1e-3) / 1e9
-    traffic = recorded_traffic(rows)
+    traffic = recorded_traffic(rows, V)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
@@ -480,7 +630,8 @@ def run_ours(args):
                      "frac_of_nominal_8TBps": achieved / 8000.0},
         "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": LAUNCHES_PER_STEP * args.steps,
         "clocks": clocks, "windowed_kl_sum": loss, "probe_pass": probe_line, "return_to_go_path": rtg_line,
-        "teacher_drift_path": drift_line,
+        "teacher_drift_path": drift_line, "config4_probe": cfg4_line, "n2_path": n2_line,
+        "lmhead_path": lm_line, "sustained": sustained,
         "L_next": int(al.L_next.item()),
     }
     print(json.dumps(line))

@@ -271,7 +271,12 @@ def lmhead_fwd_bwd(Hs, Ws, Ht, Wt, tokens, window, rollout_len=None, grad_scale:
       G[b,t,:] = d loss / d z[b,t,:] for t inside the window, zero elsewhere
       dH[b,t,:] = G[b,t,:] Ws                              chain rule through z = H_s W_s^T
       dW       += G[b]^T Hs[b]
-    Returns dict(kl, logratio, gsq, lse_s, lse_t [B,T]; dH [B,T,d_s]; dW [V,d_s]), float64.
+    Returns dict(kl, logratio, gsq, lse_s, lse_t [B,T]; dH [B,T,d_s]; dW [V,d_s]), float64, and
+    beside each gradient the sum of the absolute values of its terms, dH_abs = |G| |W_s| and
+    dW_abs = |G|^T |H_s|: the scale against which a rounding of G is bounded; and dH_cond =
+    (s P) |W_s|, dW_cond = (s P)^T |H_s| with P the student probabilities of the in-window rows
+    and s = max(1, |E_p[z - u]|) per row: the scale against which an absolute perturbation of the
+    centred difference (z_k - u_k) - E_p[z - u] inside g_k is bounded.
     """
     Hs64, Ws64, Ht64, Wt64 = widen(Hs), widen(Ws), widen(Ht), widen(Wt)
     B, T, ds = Hs64.shape
@@ -283,6 +288,10 @@ def lmhead_fwd_bwd(Hs, Ws, Ht, Wt, tokens, window, rollout_len=None, grad_scale:
     out = {k: np.zeros((B, T)) for k in ("kl", "logratio", "gsq", "lse_s", "lse_t")}
     dH = np.zeros((B, T, ds))
     dW = np.zeros((V, ds))
+    dH_abs = np.zeros((B, T, ds))
+    dW_abs = np.zeros((V, ds))
+    dH_cond = np.zeros((B, T, ds))
+    dW_cond = np.zeros((V, ds))
     for b in range(B):
         z = (Hs64[b] @ Ws64.T)[None]
         u = (Ht64[b] @ Wt64.T)[None]
@@ -293,8 +302,19 @@ def lmhead_fwd_bwd(Hs, Ws, Ht, Wt, tokens, window, rollout_len=None, grad_scale:
             out[name][b] = val[0]
         dH[b] = G[0] @ Ws64
         dW += G[0].T @ Hs64[b]
+        dH_abs[b] = np.abs(G[0]) @ np.abs(Ws64)
+        dW_abs += np.abs(G[0]).T @ np.abs(Hs64[b])
+        inside = (np.arange(T) < min(window[b], rollout_len[b]))[:, None]
+        sP = np.where(inside, np.exp(z[0] - ls[0][:, None]) *
+                      np.maximum(1.0, np.abs(kl[0] + ls[0] - lt[0]))[:, None], 0.0)
+        dH_cond[b] = sP @ np.abs(Ws64)
+        dW_cond += sP.T @ np.abs(Hs64[b])
     out["dH"] = dH
     out["dW"] = dW
+    out["dH_abs"] = dH_abs
+    out["dW_abs"] = dW_abs
+    out["dH_cond"] = dH_cond
+    out["dW_cond"] = dW_cond
     return out
 
 

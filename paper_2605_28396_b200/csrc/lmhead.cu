@@ -28,15 +28,20 @@ namespace {
 
 using namespace tc;
 
-constexpr int kRecFields = 12;   // m2s, S, A, B0, B1, B2, m2t, St, dref, zy, uy, has_y
+constexpr int kRecFields = 8;    // m2s, S, A, B0, B1, B2, m2t, St
+constexpr int kTokFields = 4;    // z_y, u_y, has_y, unused
 constexpr int kInfoFields = 8;   // L2s, a1, a0, gy, y (bits), unused x3
 constexpr int kTileFields = 8;   // b, t0, nvalid, ngrad, gidx, unused x3
-constexpr float kMasked = -1.0e30f;
+// Logit value given to the columns past the vocabulary in the last tile: far enough below any
+// real logit that its exponential is exactly zero against a real row maximum, and small enough
+// that the rounding residual of z*log2e against the running reference stays a fraction of one
+// (a partial that sees only such columns keeps finite sums and merges with weight 2^-huge = 0).
+constexpr float kMasked = -1.0e6f;
 
 // ---------------------------------------------------------------------------- workspace
 struct LmLayout {
-  size_t off_rowmap, off_hdr, off_tiles, off_g2t, off_rowdst, off_info, off_part, off_hs, off_ht,
-      off_hg, off_G, total;
+  size_t off_rowmap, off_hdr, off_tiles, off_g2t, off_rowdst, off_info, off_tok, off_part, off_hs,
+      off_ht, off_hg, off_G, total;
   int64_t max_tiles;
   int n_groups, n_chunks;
   int64_t ldG;
@@ -68,6 +73,7 @@ LmLayout lm_layout(int64_t B, int64_t T, int64_t V, int64_t ds, int64_t dt, int6
   L.off_g2t = o;     o = up(o + (size_t)L.max_tiles * 4);
   L.off_rowdst = o;  o = up(o + rows * 4);
   L.off_info = o;    o = up(o + rows * kInfoFields * 4);
+  L.off_tok = o;     o = up(o + rows * kTokFields * 4);
   L.off_part = o;    o = up(o + rows * (size_t)L.n_groups * 2 * kRecFields * 4);
   L.off_hs = o;      o = up(o + rows * (size_t)ds * 2);
   L.off_ht = o;      o = up(o + rows * (size_t)dt * 2);
@@ -190,16 +196,66 @@ __global__ void __launch_bounds__(256) lm_gather_kernel(const __nv_bfloat16* __r
   }
 }
 
+// The two logits at the sampled token of every processed position, z_y = h_s . W_s[y] and
+// u_y = h_t . W_t[y], as plain fp32 dot products (one warp per compact row).  They give the
+// sampled-token log-ratio of Section 2.3 without a search through the logit tiles, and their
+// difference is the value the sweep centres z - u on: on a peaked row the sampled token is almost
+// surely the peak, where the centred difference is then exactly zero, which keeps the
+// single-sweep squared-norm moments well conditioned.
+__device__ __forceinline__ float warp_dot_bf16(const __nv_bfloat16* a, const __nv_bfloat16* b,
+                                               int64_t d, int lane) {
+  float acc = 0.f;
+  for (int64_t v = lane; v < d / 8; v += 32) {
+    const uint4 x = reinterpret_cast<const uint4*>(a)[v], y = reinterpret_cast<const uint4*>(b)[v];
+    float xf[8], yf[8];
+    Elem<__nv_bfloat16>::unpack(x, xf);
+    Elem<__nv_bfloat16>::unpack(y, yf);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc = fmaf(xf[i], yf[i], acc);
+  }
+  return warp_sum(acc);
+}
+
+__global__ void __launch_bounds__(256) lm_token_kernel(
+    const __nv_bfloat16* __restrict__ hs_c, const __nv_bfloat16* __restrict__ ws,
+    const __nv_bfloat16* __restrict__ ht_c, const __nv_bfloat16* __restrict__ wt, int64_t T,
+    int64_t V, int64_t ds, int64_t dt, const int32_t* hdr, const int32_t* __restrict__ tiles,
+    const int32_t* __restrict__ tokens, float* tok) {
+  const int lane = threadIdx.x & 31;
+  const int64_t n_rows = (int64_t)hdr[0] * kBM;
+  for (int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); row < n_rows;
+       row += (int64_t)gridDim.x * 8) {
+    const int32_t* e = tiles + (row / kBM) * kTileFields;
+    const int i = (int)(row % kBM);
+    float zy = 0.f, uy = 0.f, has = 0.f;
+    if (i < e[2]) {
+      const int y = tokens[(int64_t)e[0] * T + e[1] + i];
+      if (y >= 0 && y < V) {
+        zy = warp_dot_bf16(hs_c + row * ds, ws + (int64_t)y * ds, ds, lane);
+        uy = warp_dot_bf16(ht_c + row * dt, wt + (int64_t)y * dt, dt, lane);
+        has = 1.f;
+      }
+    }
+    if (lane == 0) {
+      float* o = tok + row * kTokFields;
+      o[0] = zy;
+      o[1] = uy;
+      o[2] = has;
+      o[3] = 0.f;
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------- sweep kernel
 struct SweepParams {
   const int32_t* hdr;
   const int32_t* tiles;
   const int32_t* g2t;
-  const int32_t* tokens;
+  const float* tok;             // sweep 1 in: z_y, u_y per compact row
   int64_t T, V;
   int ks_blocks, kt_blocks;     // k-blocks of the student / teacher contraction
   int n_chunks, n_groups;
-  float* part;                  // sweep 1 out
+  float* part;                  // sweep 1 out: partial records; sweep 2 out: partial sum g^2
   const float* info;            // sweep 2 in
   __nv_bfloat16* G;             // sweep 2 out
   int64_t ldG;
@@ -326,21 +382,17 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
     for (int64_t item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
       const int tile_c = (int)(item / p.n_groups), g = (int)(item % p.n_groups);
       const int tile = GRAD ? p.g2t[tile_c] : tile_c;
-      const int32_t* te = p.tiles + (int64_t)tile * kTileFields;
-      const int nrow = GRAD ? te[3] : te[2];
       int c0, c1;
       group_chunks(p, g, c0, c1);
 
       int y = -1;
       RowAcc acc;
-      float dref = 0.f, zy = 0.f, uy = 0.f, has_y = 0.f;
+      float dref = 0.f, q = 0.f;   // q: this thread's share of the row's sum g^2 (sweep 2)
       float L2s = 0.f, a1 = 0.f, a0 = 0.f, gy = 0.f;
       if (!GRAD) {
         acc.reset();
-        if (row < nrow) {
-          y = p.tokens[(int64_t)te[0] * p.T + te[1] + row];
-          if (y < 0 || y >= p.V) y = -1;   // reported by the merge step; never matches a column
-        }
+        const float* tk = p.tok + ((int64_t)tile * kBM + row) * kTokFields;
+        dref = tk[0] - tk[1];      // centre of z - u for this row: the sampled token's difference
       } else {
         const float* inf = p.info + ((int64_t)tile * kBM + row) * kInfoFields;
         L2s = inf[0];
@@ -349,7 +401,6 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
         gy = inf[3];
         y = __float_as_int(inf[4]);
       }
-      bool first = true;
       for (int c = c0; ok && c < c1; ++c, ++acc_it) {
         if (!__all_sync(0xffffffffu, bar_wait(smem_addr(&ctrl->acc_full[0]), acc_it & 1, abort))) {
           ok = false;   // the same decision in every lane: tcgen05.ld below is warp-collective
@@ -371,28 +422,15 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
             z[i] = __uint_as_float(zr[i]);
             u[i] = NEED_U ? __uint_as_float(ur[i]) : 0.f;
           }
+          if (ragged) {   // columns past the vocabulary: exp -> 0, z - u -> 0
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (col + i >= p.V) {
+                z[i] = kMasked;
+                u[i] = kMasked;
+              }
+          }
           if (!GRAD) {
-            if (ragged) {
-#pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (col + i >= p.V) {
-                  z[i] = kMasked;
-                  u[i] = kMasked;
-                }
-            }
-            if (first) {
-              dref = z[0] - u[0];
-              first = false;
-            }
-            if ((unsigned)(y - (int)col) < 32u) {
-#pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (i == y - (int)col) {
-                  zy = z[i];
-                  uy = u[i];
-                }
-              has_y = 1.f;
-            }
             acc_piece<32, true>(z, u, dref, acc);
           } else {
             uint32_t pk[16];
@@ -404,6 +442,7 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
                 const float pz = ex2f(fmaf(z[i + e], kLog2e, -L2s));
                 const float w = NEED_U ? fmaf(a1, z[i + e] - u[i + e], a0) : a0;
                 gv[e] = pz * w;
+                q = fmaf(gv[e], gv[e], q);
               }
               pk[i >> 1] = pack_bf16x2(gv[0], gv[1]);
             }
@@ -415,6 +454,7 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
                   const float pz = ex2f(fmaf(z[i], kLog2e, -L2s));
                   const float w = NEED_U ? fmaf(a1, z[i] - u[i], a0) : a0;
                   const float gv = fmaf(pz, w, gy);
+                  q += gv * gv - (pz * w) * (pz * w);
                   const uint32_t h = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(gv));
                   pk[i >> 1] = (i & 1) ? ((pk[i >> 1] & 0x0000ffffu) | (h << 16))
                                        : ((pk[i >> 1] & 0xffff0000u) | h);
@@ -431,6 +471,8 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
         tc_fence_before_sync();
         bar_arrive(smem_addr(&ctrl->acc_empty[0]));
       }
+      if (GRAD && ok)
+        p.part[(((int64_t)tile_c * p.n_groups + g) * 2 + half) * kBM + row] = q;
       if (!GRAD && ok) {
         float* o = p.part + ((((int64_t)tile * p.n_groups + g) * 2 + half) * kRecFields) * kBM + row;
         o[0 * kBM] = acc.m2s;
@@ -441,10 +483,6 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
         o[5 * kBM] = acc.B2;
         o[6 * kBM] = acc.m2t;
         o[7 * kBM] = acc.St;
-        o[8 * kBM] = dref;
-        o[9 * kBM] = zy;
-        o[10 * kBM] = uy;
-        o[11 * kBM] = has_y;
       }
     }
   }
@@ -463,6 +501,7 @@ struct MergeParams {
   const int32_t* tiles;
   const int32_t* tokens;
   const float* part;
+  const float* tok;
   float* info;
   int64_t T, V;
   int n_groups;
@@ -497,24 +536,22 @@ __global__ void __launch_bounds__(kBM) lm_merge_kernel(const MergeParams p) {
     M2s = fmax(M2s, f(i, 0));
     M2t = fmax(M2t, f(i, 6));
   }
-  double S = 0, St = 0, AS = 0;
-  double zy = 0, uy = 0;
-  bool has_y = false;
+  const float* tk = p.tok + ((int64_t)tile * kBM + row) * kTokFields;
+  const bool has_y = tk[2] != 0.f;
+  const double zy = tk[0], uy = tk[1];
+  const double dref = (double)(tk[0] - tk[1]);   // the centre the sweep used (an fp32 difference)
+  double S = 0, St = 0, Ac = 0;
   for (int i = 0; i < n; ++i) {
     const double w = exp2(f(i, 0) - M2s);
     S += w * f(i, 1);
-    AS += w * (f(i, 2) + f(i, 8) * f(i, 1));
+    Ac += w * f(i, 2);
     St += exp2(f(i, 6) - M2t) * f(i, 7);
-    if (f(i, 11) != 0.0) {
-      has_y = true;
-      zy = f(i, 9);
-      uy = f(i, 10);
-    }
   }
-  const double c0 = AS / S;                    // E_p[z - u]
+  const double sh = -Ac / S;                   // centre minus E_p[z - u]
+  const double c0 = dref - sh;                 // E_p[z - u]
   double B0 = 0, B2c = 0;
   for (int i = 0; i < n; ++i) {
-    const double w = exp2(f(i, 0) - M2s), w2 = w * w, sh = f(i, 8) - c0;
+    const double w = exp2(f(i, 0) - M2s), w2 = w * w;
     B0 += w2 * f(i, 3);
     B2c += w2 * (f(i, 5) + 2.0 * sh * f(i, 4) + sh * sh * f(i, 3));
   }
@@ -552,6 +589,22 @@ __global__ void __launch_bounds__(kBM) lm_merge_kernel(const MergeParams p) {
   inf[4] = __int_as_float(in_grad && has_y ? p.tokens[r] : -1);
   if (!has_y) atomicOr(p.status, ADWIN_DEV_TOKEN_RANGE);
   if (!(isfinite(lse_s) && isfinite(lse_t))) atomicOr(p.status, ADWIN_DEV_NONFINITE);
+}
+
+// Squared gradient norm of the rows whose gradient sweep 2 formed: the sum of g_k^2 over the
+// entries themselves (fixed order, float64), which replaces the single-sweep moment value there.
+__global__ void __launch_bounds__(kBM) lm_gsq_kernel(const int32_t* hdr, const float* __restrict__ part,
+                                                     const int32_t* __restrict__ rowdst,
+                                                     int n_groups, float* gsq) {
+  const int gt = blockIdx.x;
+  if (gt >= hdr[1]) return;
+  const int row = threadIdx.x;
+  const int32_t dst = rowdst[(int64_t)gt * kBM + row];
+  if (dst < 0) return;
+  double acc = 0.0;
+  for (int i = 0; i < n_groups * 2; ++i)
+    acc += (double)part[((int64_t)gt * n_groups * 2 + i) * kBM + row];
+  gsq[dst] = (float)acc;
 }
 
 // ---------------------------------------------------------------------------- GEMM kernel
@@ -785,6 +838,7 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
   int32_t* g2t = reinterpret_cast<int32_t*>(wb + L.off_g2t);
   int32_t* rowdst = reinterpret_cast<int32_t*>(wb + L.off_rowdst);
   float* info = reinterpret_cast<float*>(wb + L.off_info);
+  float* tok = reinterpret_cast<float*>(wb + L.off_tok);
   float* part = reinterpret_cast<float*>(wb + L.off_part);
   __nv_bfloat16* hs_c = reinterpret_cast<__nv_bfloat16*>(wb + L.off_hs);
   __nv_bfloat16* ht_c = reinterpret_cast<__nv_bfloat16*>(wb + L.off_ht);
@@ -807,6 +861,9 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
   if (want_grad && range_full)
     lm_gather_kernel<<<gather_blocks, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(hs), T, ds,
                                                    hdr, tiles, g2t, true, hs_g);
+  lm_token_kernel<<<gather_blocks, 256, 0, s>>>(hs_c, static_cast<const __nv_bfloat16*>(ws), ht_c,
+                                                static_cast<const __nv_bfloat16*>(wt), T, V, ds, dt,
+                                                hdr, tiles, tokens, tok);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
   CUtensorMap m_hs, m_ws, m_ht, m_wt;
@@ -818,7 +875,7 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
   sp.hdr = hdr;
   sp.tiles = tiles;
   sp.g2t = g2t;
-  sp.tokens = tokens;
+  sp.tok = tok;
   sp.T = T;
   sp.V = V;
   sp.ks_blocks = (int)((ds + kBK - 1) / kBK);
@@ -839,6 +896,7 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
   mp.tiles = tiles;
   mp.tokens = tokens;
   mp.part = part;
+  mp.tok = tok;
   mp.info = info;
   mp.T = T;
   mp.V = V;
@@ -870,6 +928,7 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
     if ((e = opt_in_smem(lm_sweep_kernel<true, false>)) != cudaSuccess) return e;
     lm_sweep_kernel<true, false><<<sm_count, kThreads, kSmemBytes, s>>>(m_hg, m_ws, m_ht, m_wt, sp);
   }
+  if (gsq) lm_gsq_kernel<<<(unsigned)L.max_tiles, kBM, 0, s>>>(hdr, part, rowdst, L.n_groups, gsq);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
   if (dH) {
