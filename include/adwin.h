@@ -323,6 +323,9 @@ int adwin_opd_kl_fwd_bwd_host(const void* student_host, const void* teacher_host
  * `workspace` / `workspace_bytes` left out.  Differences:
  *   - B may be at most adwin_no_alloc_max_sequences() (4096); a larger batch returns
  *     ADWIN_ERR_WORKSPACE and enqueues nothing.  T and V are not limited by the array.
+ *   - The array has room for the second set of prefix sums (the one that lets an
+ *     ADWIN_RANGE_FULL call with gradient run as two kernels) only up to B = 2719; above that
+ *     such a call runs as one kernel, with the same results to within rounding order.
  *   - The first call on each device looks up the array's device address (that device must be
  *     current, as for every call).  Make that first call outside any stream capture.
  *   - All calls on a device share the one array.  Each call rewrites it completely before reading

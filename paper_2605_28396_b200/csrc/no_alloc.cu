@@ -58,10 +58,10 @@ int adwin_opd_kl_fwd_bwd_no_alloc(const void* student_logits, const void* teache
   if (B > 0 && workspace_layout(B).total > kScratchBytes) return ADWIN_ERR_WORKSPACE;
   void* scratch = scratch_for_current_device();
   if (scratch == nullptr) return ADWIN_ERR_CUDA;
-  // Every call rewrites the whole row map before any kernel reads it, so nothing a previous call
-  // left behind is ever used; the header block, which no kernel writes, is put back to zero.
-  if (cudaMemsetAsync(scratch, 0, 256, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
-    return ADWIN_ERR_CUDA;
+  // Nothing in the array has to start at zero: the row-map kernel of every call rewrites all the
+  // entries that the call's other kernels read before they read them (the 256-byte header is
+  // reserved and neither read nor written), so nothing a previous call left behind is ever used.
+  // Nothing is enqueued here either: the ordinary entry point validates the arguments first.
   return adwin_opd_kl_fwd_bwd(student_logits, teacher_logits, dtype, B, T, V, ld, tokens, window,
                               rollout_len, grad_scale, grad_mode, flags, grad_student, grad_dtype,
                               ld_grad, kl, logratio, gsq, lse_student, lse_teacher, scratch,

@@ -129,6 +129,20 @@ def test_sampled_token_far_below_the_row_maximum(path, in_dt, g_dt):
     run_and_check(batch, grad_dtype=g_dt, grad_mode=api.GRAD_SAMPLED, flags=flags)
 
 
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("in_dt,g_dt,shift", [(1, torch.float32, 50.0), (2, torch.bfloat16, 50.0),
+                                              (2, torch.bfloat16, 1000.0), (2, None, 1000.0)])
+def test_teacher_rows_shifted_by_a_constant(path, in_dt, g_dt, shift):
+    """The divergence does not depend on a constant added to a logit row.  The kernels work with
+    z - u, which such an offset makes large against the differences that matter; an offset of 50
+    must stay inside the fp32 tolerance, one of 1000 inside the bf16 tolerance."""
+    batch = synth.make_batch(in_dt, device=DEV, B=2, T=10, V=8192)
+    batch.window = torch.tensor([10, 6], dtype=torch.int32, device=DEV)
+    batch.teacher = (batch.teacher.float() + shift).to(batch.teacher.dtype)
+    for mode in (api.GRAD_FULL_KL, api.GRAD_SAMPLED):
+        run_and_check(batch, grad_dtype=g_dt, grad_mode=mode, flags=PATHS[path])
+
+
 @pytest.mark.parametrize("g_dt", [torch.bfloat16, None])
 def test_teacher_logits_outside_the_range_of_the_polynomial_exponential(g_dt):
     """The staged kernel takes the exponential of the first teacher pair of every 16-byte piece
