@@ -82,6 +82,19 @@ enum {
 /* Library ABI version (bumped when a signature changes). */
 int adwin_version(void);
 
+/*
+ * Diagnostic.  Every on-chip wait of the kernels (a consumer waiting for a bulk copy, a producer
+ * for a free slot, the exchange between the CTAs of a cluster, the epilogue for an accumulator) is
+ * bounded: when it runs out the kernel raises ADWIN_DEV_TIMEOUT, stops waiting anywhere, waits
+ * for its own copies and MMAs in flight (those waits keep the full limit), frees its tensor
+ * memory and returns; the outputs of that call are invalid, the context stays usable.  This sets
+ * the limit of those handshake waits for the launches that follow, process-wide, in nanoseconds
+ * (default 2 s; 0 restores the default).  A limit of a few nanoseconds makes the first wait that
+ * is not already satisfied run out, which is how the tests exercise the give-up path; there is
+ * no other use for it.  The paper has no counterpart.
+ */
+void adwin_diag_set_wait_limit_ns(uint64_t ns);
+
 /* Human-readable name of an adwin_status_t.  Host pointer to a static string. */
 const char* adwin_status_string(int status);
 

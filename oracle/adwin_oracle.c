@@ -441,6 +441,85 @@ void adwin_oracle_topk_survival(const int64_t *rank, const int32_t *rollout_len,
   }
 }
 
+/*
+ * Scale of the terms that a ONE-sweep evaluation of gsq adds and subtracts (a conditioning
+ * measure for tests, not a quantity of the method).  Without a second sweep the squared norm
+ * sum_k p_k^2 (delta_k - E_p delta)^2, delta = z - u, can only be accumulated about a centre that
+ * is known beforehand -- the sampled token's delta_y -- and corrected afterwards:
+ *   sum p^2 (delta - delta_y)^2 - 2 c0 sum p^2 (delta - delta_y) + c0^2 sum p^2,  c0 = E_p delta - delta_y.
+ * Each of the three sums is bounded by  2 sum_k p_k^2 [ (delta_k - delta_y)^2 + c0^2 ],  which is what
+ * this returns (times alpha^2).  On a peaked row with an off-peak sample it exceeds gsq by orders
+ * of magnitude, and a float32 evaluation then keeps correspondingly fewer digits of gsq.
+ * SAMPLED mode: gsq = (alpha c)^2 [ (1 - p_y)^2 + sum_{k != y} p_k^2 ] is evaluated as
+ * sum p^2 - p_y^2 + (1 - p_y)^2; the scale returned is (alpha c)^2 [ sum p^2 + p_y^2 + (1 - p_y)^2 ].
+ * y outside [0,V): the centre is delta_0 (FULL_KL), the result NaN (SAMPLED).
+ */
+double adwin_oracle_gsq_term_scale(const double *z, const double *u, int64_t V, int64_t y,
+                                   double alpha, int mode) {
+  double ls = adwin_oracle_logsumexp(z, V);
+  double lt = adwin_oracle_logsumexp(u, V);
+  int ok = (y >= 0 && y < V);
+  double dy = ok ? z[y] - u[y] : z[0] - u[0];
+  double mean = 0.0, mc = 0.0;
+  for (int64_t k = 0; k < V; ++k) comp_add(&mean, &mc, exp(z[k] - ls) * (z[k] - u[k]));
+  double c0 = (mean + mc) - dy;
+  double acc = 0.0, comp = 0.0, p2 = 0.0, p2c = 0.0;
+  for (int64_t k = 0; k < V; ++k) {
+    double p = exp(z[k] - ls);
+    double d = (z[k] - u[k]) - dy;
+    comp_add(&acc, &comp, p * p * (d * d + c0 * c0));
+    comp_add(&p2, &p2c, p * p);
+  }
+  if (mode == ORACLE_MODE_FULL_KL) return 2.0 * alpha * alpha * (acc + comp);
+  if (!ok) return NAN;
+  double py = exp(z[y] - ls);
+  double c = (z[y] - ls) - (u[y] - lt);
+  return alpha * alpha * c * c * ((p2 + p2c) + py * py + (1.0 - py) * (1.0 - py));
+}
+
+/* The same for every processed position of a batch (0 elsewhere); arguments as in
+ * adwin_oracle_opd_kl_fwd_bwd. */
+int adwin_oracle_gsq_term_scale_batch(const void *student, const void *teacher, int dtype,
+                                      int64_t B, int64_t T, int64_t V, int64_t ld,
+                                      const int32_t *tokens, const int32_t *window,
+                                      const int32_t *rollout_len, double grad_scale, int grad_mode,
+                                      int flags, double *scale) {
+  for (int64_t b = 0; b < B; ++b) {
+    int64_t R = rollout_len ? rollout_len[b] : T;
+    if (window[b] < 0 || R < 0 || R > T) return 5;
+  }
+  int64_t rows = B * T;
+#ifdef _OPENMP
+#pragma omp parallel
+#endif
+  {
+    double *z = (double *)malloc(sizeof(double) * (size_t)(V > 0 ? V : 1));
+    double *u = (double *)malloc(sizeof(double) * (size_t)(V > 0 ? V : 1));
+#ifdef _OPENMP
+#pragma omp for schedule(dynamic, 1)
+#endif
+    for (int64_t r = 0; r < rows; ++r) {
+      int64_t b = r / T, t = r % T;
+      int64_t R = rollout_len ? rollout_len[b] : T;
+      int in_window = (t < window[b]) && (t < R) && (t < T);
+      int in_rollout = (t < R) && (t < T);
+      int processed = (flags & ORACLE_FLAG_RANGE_FULL) ? in_rollout : in_window;
+      double v = 0.0;
+      if (processed) {
+        for (int64_t k = 0; k < V; ++k) {
+          z[k] = load_logit(student, dtype, r * ld + k);
+          u[k] = load_logit(teacher, dtype, r * ld + k);
+        }
+        v = adwin_oracle_gsq_term_scale(z, u, V, tokens[r], grad_scale, grad_mode);
+      }
+      scale[r] = v;
+    }
+    free(z);
+    free(u);
+  }
+  return 0;
+}
+
 int adwin_oracle_num_threads(void) {
 #ifdef _OPENMP
   extern int omp_get_max_threads(void);

@@ -47,6 +47,8 @@ def lib():
         L.adwin_oracle_literal_cosine.restype = ctypes.c_double
         L.adwin_oracle_opd_kl_fwd_bwd.restype = ctypes.c_int
         L.adwin_oracle_num_threads.restype = ctypes.c_int
+        L.adwin_oracle_gsq_term_scale.restype = ctypes.c_double
+        L.adwin_oracle_gsq_term_scale_batch.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -129,6 +131,32 @@ def opd_kl_fwd_bwd(student, teacher, tokens, window, rollout_len=None, grad_scal
     if rc != 0:
         raise ValueError(f"oracle rejected window / rollout lengths (code {rc})")
     return dict(kl=kl, logratio=c, gsq=gsq, lse_s=ls, lse_t=lt, grad=grad)
+
+
+def gsq_term_scale(student, teacher, tokens, window, rollout_len=None, grad_scale: float = 1.0,
+                   grad_mode: int = MODE_FULL_KL, flags: int = 0):
+    """Conditioning scale of a one-sweep evaluation of gsq, per processed position ([B,T] float64):
+    the magnitude of the terms such an evaluation adds and subtracts (see the C function)."""
+    s, dt = _logit_array(student)
+    t, dt2 = _logit_array(teacher)
+    assert dt == dt2 and s.shape == t.shape and s.ndim == 3
+    B, T, V = s.shape
+    tokens, window, rollout_len = _i32(tokens), _i32(window), _i32(rollout_len)
+    out = np.empty((B, T), dtype=np.float64)
+    rc = lib().adwin_oracle_gsq_term_scale_batch(
+        _p(s), _p(t), ctypes.c_int(dt), ctypes.c_int64(B), ctypes.c_int64(T), ctypes.c_int64(V),
+        ctypes.c_int64(V), _p(tokens), _p(window), _p(rollout_len), ctypes.c_double(grad_scale),
+        ctypes.c_int(grad_mode), ctypes.c_int(flags), _p(out))
+    if rc != 0:
+        raise ValueError(f"oracle rejected window / rollout lengths (code {rc})")
+    return out
+
+
+def row_gsq_term_scale(z, u, y: int, alpha: float = 1.0, mode: int = MODE_FULL_KL) -> float:
+    z, u = _f64(z), _f64(u)
+    return float(lib().adwin_oracle_gsq_term_scale(_p(z), _p(u), ctypes.c_int64(z.size),
+                                                   ctypes.c_int64(int(y)), ctypes.c_double(alpha),
+                                                   ctypes.c_int(mode)))
 
 
 def window_reduce(kl, logratio, gsq, window, rollout_len=None):

@@ -29,7 +29,8 @@ EXPORTS = ("adwin_version", "adwin_status_string", "adwin_workspace_bytes",
            "adwin_host_staging_bytes", "adwin_opd_kl_fwd_bwd_host",
            "adwin_no_alloc_max_sequences", "adwin_opd_kl_fwd_bwd_no_alloc",
            "adwin_return_to_go", "adwin_opd_kl_fwd_bwd_weighted", "adwin_teacher_drift",
-           "adwin_drift_curves", "adwin_lmhead_workspace_bytes", "adwin_opd_kl_lmhead_fwd_bwd")
+           "adwin_drift_curves", "adwin_lmhead_workspace_bytes", "adwin_opd_kl_lmhead_fwd_bwd",
+           "adwin_diag_set_wait_limit_ns")
 
 _lib = None
 
@@ -38,6 +39,14 @@ class AdwinError(RuntimeError):
     def __init__(self, code: int):
         self.code = code
         super().__init__(lib().adwin_status_string(code).decode())
+
+
+def use_library(path=None):
+    """Bind the calls to another build of the library (the bounds-checked flavour
+    ``libadwin_b200_checked.so``), or back to the default one with ``path=None``."""
+    global _lib, LIB_PATH
+    LIB_PATH = Path(path) if path is not None else _PKG / "libadwin_b200.so"
+    _lib = None
 
 
 def lib():
@@ -96,6 +105,8 @@ def lib():
                                                   vp, f32, ctypes.c_int, ctypes.c_int, vp,
                                                   ctypes.c_int, vp, vp, vp, vp, vp, vp, i64, vp,
                                                   sz, vp, vp]
+        L.adwin_diag_set_wait_limit_ns.restype = None
+        L.adwin_diag_set_wait_limit_ns.argtypes = [ctypes.c_uint64]
         _lib = L
     return _lib
 
@@ -412,3 +423,8 @@ def adwin_opd_kl_lmhead_fwd_bwd(hidden_student, w_student, hidden_teacher, w_tea
         _stream(dev)))
     return SimpleNamespace(kl=kl, logratio=logratio, gsq=gsq, lse_s=lse_s, lse_t=lse_t,
                            dev_status=dev_status, workspace=workspace)
+
+
+def adwin_diag_set_wait_limit_ns(ns: int) -> None:
+    """Diagnostic: limit of the kernels' handshake waits for the launches that follow (0 = default)."""
+    lib().adwin_diag_set_wait_limit_ns(int(ns))

@@ -1,11 +1,16 @@
 // extern "C" entry points: argument validation and kernel dispatch.  No allocation, no
 // synchronisation; everything is enqueued on the caller's stream.
+#include <atomic>
 #include <mutex>
 
 #include "adwin_common.cuh"
 #include "adwin_internal.h"
 
 namespace adwin {
+
+static std::atomic<uint64_t> g_handshake_limit_ns{2000000000ull};
+uint64_t handshake_wait_limit_ns() { return g_handshake_limit_ns.load(); }
+
 namespace {
 
 constexpr int kKnownFlags =
@@ -49,7 +54,11 @@ using namespace adwin;
 
 extern "C" {
 
-int adwin_version(void) { return 1; }
+int adwin_version(void) { return 2; }
+
+void adwin_diag_set_wait_limit_ns(uint64_t ns) {
+  g_handshake_limit_ns.store(ns == 0 ? 2000000000ull : ns);
+}
 
 const char* adwin_status_string(int status) {
   switch (status) {

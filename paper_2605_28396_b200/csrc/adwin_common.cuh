@@ -18,6 +18,21 @@ namespace adwin {
 
 constexpr float kLog2e = 1.4426950408889634f;
 
+// Bounds-checked build flavour (-DADWIN_CHECKED; compute-sanitizer's stand-in): every index the
+// kernels form by hand -- shared-memory slots, ring cursors, exchange records, global pieces -- is
+// tested before the access; a violation skips the access and raises ADWIN_DEV_BOUNDS in the status
+// word.  Nothing traps.  In the ordinary build ADWIN_CHK(cond, status) is the constant `true` and
+// the test disappears.  Usage:  if (ADWIN_CHK(i < n, p.status)) { ... a[i] ... }
+#ifdef ADWIN_CHECKED
+__device__ __forceinline__ bool chk_in_bounds(bool ok, int32_t* status) {
+  if (!ok) atomicOr(status, (int32_t)ADWIN_DEV_BOUNDS);
+  return ok;
+}
+#define ADWIN_CHK(cond, status) (::adwin::chk_in_bounds((cond), (status)))
+#else
+#define ADWIN_CHK(cond, status) (true)
+#endif
+
 // Everything the row kernels need; plain pointers, filled by the host entry point.
 struct KlParams {
   const void* student;

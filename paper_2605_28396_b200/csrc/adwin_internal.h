@@ -10,6 +10,11 @@ namespace adwin {
 
 struct KlParams;
 
+// Time limit of the kernels' handshake waits (consumer / producer / exchange / accumulator
+// barriers), 2 s unless the diagnostic entry point shortened it.  The loops that wait for a
+// kernel's own copies or MMAs in flight on its way out always keep the 2 s limit.
+uint64_t handshake_wait_limit_ns();
+
 // Workspace layout: [0,256) reserved counters; offsets (B+1) int64; range B int32; ewin B int32:
 // `total` bytes, the part every call needs.  Optional extension up to `total_ext`: a second
 // prefix-sum array over the effective windows, offsets_win (B+1) int64, which lets a call that

@@ -107,6 +107,7 @@ __global__ void __launch_bounds__(kGenericThreads) kl_generic_kernel(KlParams p)
       for (; i + (kGenericUnroll - 1) * kGenericThreads < pieces;
            i += kGenericUnroll * kGenericThreads) {
         uint4 zv[kGenericUnroll], uv[kGenericUnroll];
+        if (!ADWIN_CHK(i + (kGenericUnroll - 1) * kGenericThreads < pieces && (i + (kGenericUnroll - 1) * kGenericThreads + 1) * N <= p.ld, p.status)) break;
 #pragma unroll
         for (int h = 0; h < kGenericUnroll; ++h) {
           zv[h] = write_grad ? __ldg(zs + i + h * kGenericThreads) : __ldcs(zs + i + h * kGenericThreads);
@@ -122,6 +123,7 @@ __global__ void __launch_bounds__(kGenericThreads) kl_generic_kernel(KlParams p)
       }
       for (; i < pieces; i += kGenericThreads) {
         float z[N], u[N];
+        if (!ADWIN_CHK((i + 1) * N <= p.ld, p.status)) break;
         const uint4 zv = write_grad ? __ldg(zs + i) : __ldcs(zs + i);
         const uint4 uv = write_grad ? __ldg(us + i) : __ldcs(us + i);
         Elem<TIn>::unpack(zv, reinterpret_cast<float(&)[Elem<TIn>::N]>(z));
@@ -131,6 +133,7 @@ __global__ void __launch_bounds__(kGenericThreads) kl_generic_kernel(KlParams p)
     } else {
       for (int64_t i = tid; i < pieces; i += kGenericThreads) {
         float z[N], u[N];
+        if (!ADWIN_CHK(i < p.ld, p.status)) break;
         z[0] = Elem<TIn>::load1(zrow, i);
         u[0] = Elem<TIn>::load1(urow, i);
         acc_piece<N, true>(z, u, dref, a);
@@ -149,6 +152,7 @@ __global__ void __launch_bounds__(kGenericThreads) kl_generic_kernel(KlParams p)
       const bool full = (p.mode == ADWIN_GRAD_FULL_KL);
       for (int64_t i = tid; i < pieces; i += kGenericThreads) {
         float z[N], u[N], g[N];
+        if (!ADWIN_CHK((i + 1) * N <= p.V && (i + 1) * N <= p.ld_grad && (i + 1) * N <= p.ld, p.status)) break;
         if (VEC) {
           const uint4 zv = __ldg(reinterpret_cast<const uint4*>(zrow) + i);
           const uint4 uv = __ldg(reinterpret_cast<const uint4*>(urow) + i);
@@ -201,7 +205,7 @@ __global__ void __launch_bounds__(kGenericThreads) kl_generic_kernel(KlParams p)
 #pragma unroll
       for (int w = 0; w < kGenericWarps; ++w) q += sm.wq[w];
     }
-    if (tid == 0) {
+    if (tid == 0 && ADWIN_CHK(r >= 0 && r < rows, p.status)) {
       p.kl[r] = rs.kl;
       p.logratio[r] = rs.c;
       if (p.gsq) p.gsq[r] = write_grad ? q : rs.gsq_expanded;

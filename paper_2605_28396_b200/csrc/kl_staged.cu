@@ -72,6 +72,7 @@ struct StagedPlan {
   int per_rank_pieces;    // pieces per slice (last rank may own fewer)
   int num_clusters;
   uint32_t slot_bytes;    // 2 * chunk_pieces * 16
+  uint64_t wait_limit_ns; // limit of the handshake waits (the drain loops keep kWaitLimitNs)
 };
 
 // What the consumers need to know about a row: which global row it is, whether its gradient is
@@ -201,22 +202,33 @@ __device__ __forceinline__ uint64_t global_timer() {
   return t;
 }
 
-// Bounded wait.  Returns immediately (false) once the CTA has given up.
+// Bounded wait of one thread.  Returns immediately (false) once the CTA has given up.
 template <bool CLUSTER>
-__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+__device__ __forceinline__ bool bounded_wait_lane(uint32_t bar, uint32_t parity,
+                                                  volatile int* abort, uint64_t limit_ns) {
   if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
   if (*abort) return false;
   const uint64_t t0 = global_timer();
   for (;;) {
+    // the limit is tested before each batch of polls, so that a limit shorter than one poll gives
+    // up at the first wait that is not already satisfied
+    if (global_timer() - t0 > limit_ns) {
+      *abort = 1;
+      return false;
+    }
 #pragma unroll 1
     for (int i = 0; i < 64; ++i)
       if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
     if (*abort) return false;
-    if (global_timer() - t0 > kWaitLimitNs) {
-      *abort = 1;
-      return false;
-    }
   }
+}
+// The same for a whole (converged) consumer warp: every lane polls, and the warp takes ONE
+// decision -- if any lane gave up, all do -- so that the warp-collective shuffles that follow a
+// wait are never entered by a part of the warp only.
+template <bool CLUSTER>
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile int* abort,
+                                             uint64_t limit_ns) {
+  return __all_sync(0xffffffffu, bounded_wait_lane<CLUSTER>(bar, parity, abort, limit_ns)) != 0;
 }
 
 // Walks the compact list of processed rows.  The prefix sums of the current sequence are cached
@@ -515,6 +527,17 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
     } else {
       const size_t goff = ((size_t)r * p.ld + (size_t)piece0 * N) * sizeof(TIn) +
                           (size_t)j * plan.chunk_pieces * 16;
+      // checked flavour: the copy lies inside the row's V elements and inside one slot
+      if (!ADWIN_CHK(r >= 0 && r < p.B * p.T &&
+                         ((size_t)piece0 * N) * sizeof(TIn) + (size_t)j * plan.chunk_pieces * 16 + bytes <=
+                             (size_t)p.V * sizeof(TIn) &&
+                         bytes <= u_off && 2u * u_off <= plan.slot_bytes &&
+                         slot >= res_base &&
+                         slot + plan.slot_bytes <= res_base + (size_t)(nres + nring) * plan.slot_bytes,
+                     p.status)) {
+        mbar_arrive(bar);   // keep the pipeline moving: the consumers see an empty fill
+        return;
+      }
       mbar_arrive_expect_tx(bar, 2u * bytes);
       const uint32_t dst = smem_u32(slot);
       bulk_load_hint(dst, static_cast<const char*>(p.student) + goff, bytes, bar, pol);
@@ -538,7 +561,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
         for (int j = j0; j < j1 && !stop; ++j) {
           if (ctrl.tab[j] >= 0) continue;
           if (fills >= nring &&
-              !bounded_wait<false>(smem_u32(&ctrl.ring_empty[slot]), phase ^ 1u, abort)) {
+              !bounded_wait_lane<false>(smem_u32(&ctrl.ring_empty[slot]), phase ^ 1u, abort, plan.wait_limit_ns)) {
             stop = true;   // gave up: never overwrite a slot that may still be read
             return;
           }
@@ -599,7 +622,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
           const int k = ctrl.tab[j];
           if (k < 0) continue;
           if (i > 0 &&
-              !bounded_wait<false>(smem_u32(&ctrl.res_empty[k]), (uint32_t)((i - 1) & 1), abort))
+              !bounded_wait_lane<false>(smem_u32(&ctrl.res_empty[k]), (uint32_t)((i - 1) & 1), abort, plan.wait_limit_ns))
             break;   // gave up: never overwrite a slot that may still be read
           issue_chunk(r, j, res_base + (size_t)k * plan.slot_bytes, &ctrl.res_full[k], pol_once);
           last_row = i;
@@ -627,14 +650,15 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
     for (int64_t i = 0; i < my_rows && !*abort; ++i) {
       const int ms = (int)(i % kMetaDepth);
       if (i >= kMetaDepth &&
-          !bounded_wait<false>(smem_u32(&ctrl.meta_empty[ms]),
-                               (uint32_t)((i / kMetaDepth - 1) & 1), abort))
+          !bounded_wait_lane<false>(smem_u32(&ctrl.meta_empty[ms]),
+                               (uint32_t)((i / kMetaDepth - 1) & 1), abort, plan.wait_limit_ns))
         break;
       bool wg;
       const int64_t r = cur.locate(p, cluster_id + i * plan.num_clusters, wg);
       const int y = p.tokens[r];
       float zy, uy;
       fetch_logits_at<TIn>(p, r, y, zy, uy);
+      if (!ADWIN_CHK(ms >= 0 && ms < kMetaDepth && r >= 0 && r < p.B * p.T, p.status)) break;
       RowMeta& m = ctrl.meta[ms];
       m.r = r;
       m.y = y;
@@ -672,7 +696,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       if (real) {
         const int ms = (int)(i % kMetaDepth);
         if (!bounded_wait<false>(smem_u32(&ctrl.meta_full[ms]),
-                                 (uint32_t)((i / kMetaDepth) & 1), abort)) {
+                                 (uint32_t)((i / kMetaDepth) & 1), abort, plan.wait_limit_ns)) {
           timed_out = true;
           break;
         }
@@ -708,7 +732,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
               v4 = lane_sum(hsum2(a.B1));
               v5 = lane_sum(hsum2(a.B2));
             }
-            if (lane < cl) {
+            if (lane < cl && ADWIN_CHK((int)rank * kNW + warp < kMaxRec && cl <= kMaxCL, p.status)) {
               const uint32_t dst =
                   map_to_rank(smem_u32(&ctrl.xbuf[par][rank * kNW + warp][0]), (uint32_t)lane);
               remote_store4(dst, v0s, v1, v2, v3);
@@ -720,7 +744,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
             // from here on: row i+1
             const int msn = (int)((i + 1) % kMetaDepth);
             if (!bounded_wait<false>(smem_u32(&ctrl.meta_full[msn]),
-                                     (uint32_t)(((i + 1) / kMetaDepth) & 1), abort)) {
+                                     (uint32_t)(((i + 1) / kMetaDepth) & 1), abort, plan.wait_limit_ns)) {
               timed_out = true;
               break;
             }
@@ -733,13 +757,17 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
           }
           if (v >= vend) break;   // (reached only when the leading chunks of row i+1 are done)
           const int j = v < nch ? v : v - nch;
+          if (!ADWIN_CHK(j >= 0 && j < nch && j < kMaxChunks && rc_slot >= 0 && rc_slot < nring + (nring == 0), p.status)) {
+            timed_out = true;
+            break;
+          }
           const int k = ctrl.tab[j];
           const char* sl;
           if (k >= 0) {   // resident chunks only occur in the part of row i (v < nch)
-            if (!bounded_wait<false>(smem_u32(&ctrl.res_full[k]), rpar, abort)) timed_out = true;
+            if (!bounded_wait<false>(smem_u32(&ctrl.res_full[k]), rpar, abort, plan.wait_limit_ns)) timed_out = true;
             sl = res_base + (size_t)k * plan.slot_bytes + toff;
           } else {
-            if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort)) timed_out = true;
+            if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort, plan.wait_limit_ns)) timed_out = true;
             sl = ring_base + (size_t)rc_slot * plan.slot_bytes + toff;
           }
           if (timed_out) break;
@@ -749,7 +777,8 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
           uint4 zr[kP], ur[kP];
 #pragma unroll
           for (int h = 0; h < kP; ++h) {
-            if (gt + h * kGT < np) {
+            if (gt + h * kGT < np &&
+                ADWIN_CHK(k < nres && toff + (uint32_t)(h * kGT * 16) + 16u <= u_off, p.status)) {
               zr[h] = *reinterpret_cast<const uint4*>(sl + h * kGT * 16);
               ur[h] = *reinterpret_cast<const uint4*>(sl + u_off + h * kGT * 16);
             }
@@ -783,7 +812,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       RowTotals t;
       float qtot;
       {
-        if (!bounded_wait<true>(smem_u32(&ctrl.xbar[par]), (uint32_t)((i >> 1) & 1), abort)) {
+        if (!bounded_wait<true>(smem_u32(&ctrl.xbar[par]), (uint32_t)((i >> 1) & 1), abort, plan.wait_limit_ns)) {
           timed_out = true;
           break;
         }
@@ -838,7 +867,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
           remote_store4(dst + 16, w4, w5, wmt, w7);
           remote_arrive_release(map_to_rank(smem_u32(&ctrl.sbar), (uint32_t)lane));
         }
-        if (!bounded_wait<true>(smem_u32(&ctrl.sbar), safe_rounds & 1u, abort)) {
+        if (!bounded_wait<true>(smem_u32(&ctrl.sbar), safe_rounds & 1u, abort, plan.wait_limit_ns)) {
           timed_out = true;
           break;
         }
@@ -903,7 +932,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
             if (k >= 0) {
               sl = res_base + (size_t)k * plan.slot_bytes + toff;   // still there since sweep 1
             } else {
-              if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort)) timed_out = true;
+              if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort, plan.wait_limit_ns)) timed_out = true;
               sl = ring_base + (size_t)rc_slot * plan.slot_bytes + toff;
             }
             if (timed_out) break;
@@ -911,7 +940,9 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
             uint4 zr[kP], ur[kP];
 #pragma unroll
             for (int h = 0; h < kP; ++h) {
-              if (gt + h * kGT < np) {
+              if (gt + h * kGT < np &&
+                  ADWIN_CHK(k < nres && rc_slot < nring + (nring == 0) &&
+                                toff + (uint32_t)(h * kGT * 16) + 16u <= u_off, p.status)) {
                 zr[h] = *reinterpret_cast<const uint4*>(sl + h * kGT * 16);
                 ur[h] = *reinterpret_cast<const uint4*>(sl + u_off + h * kGT * 16);
               }
@@ -952,11 +983,14 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
                 }
 #pragma unroll
                 for (int e = 0; e < NP; ++e) Q = fma2(G[e], G[e], Q);
-                store_pairs<TOut, NP>(gthread + (size_t)j * gstep + (size_t)h * kGT * N * sizeof(TOut), G);
+                // checked flavour: the 16-byte (or 32-byte) store lies inside the row's V entries
+                if (ADWIN_CHK((piece0 + (int64_t)j * plan.chunk_pieces + gt + h * kGT + 1) * N <= p.V &&
+                                  rC >= 0 && rC < p.B * p.T, p.status))
+                  store_pairs<TOut, NP>(gthread + (size_t)j * gstep + (size_t)h * kGT * N * sizeof(TOut), G);
               }
             }
           } else if (k < 0) {
-            if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort)) {
+            if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort, plan.wait_limit_ns)) {
               timed_out = true;
               break;
             }
@@ -1155,6 +1189,7 @@ cudaError_t launch_staged_t(const KlParams& p, int dtype, int grad_dtype, int sm
   cfg.numAttrs = 1;
   const int64_t rows = p.B * p.T;
   if (plan.num_clusters > rows) plan.num_clusters = (int)rows;
+  plan.wait_limit_ns = handshake_wait_limit_ns();
   cfg.gridDim = dim3(plan.cl * plan.num_clusters);
   return cudaLaunchKernelEx(&cfg, kernel, p, plan);
 }

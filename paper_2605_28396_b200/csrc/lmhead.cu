@@ -156,6 +156,7 @@ __global__ void __launch_bounds__(1024) lm_plan_kernel(const int32_t* __restrict
       const int nvalid = P - t0 < kBM ? P - t0 : kBM;
       int ngrad = E - t0;
       ngrad = ngrad < 0 ? 0 : (ngrad > kBM ? kBM : ngrad);
+      if (!ADWIN_CHK(tile < max_tiles && gt < max_tiles, status)) break;
       int32_t* e = tiles + tile * kTileFields;
       e[0] = (int32_t)b;
       e[1] = t0;
@@ -259,6 +260,8 @@ struct SweepParams {
   const float* info;            // sweep 2 in
   __nv_bfloat16* G;             // sweep 2 out
   int64_t ldG;
+  int64_t max_tiles;            // capacity of the per-tile buffers (checked flavour)
+  uint64_t limit_ns;            // limit of the handshake waits
   int32_t* status;
 };
 
@@ -323,7 +326,7 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
             const int nk = pass ? p.kt_blocks : p.ks_blocks;
             for (int kb = 0; kb < nk; ++kb, ++it) {
               const uint32_t s = it % kStages, ph = (it / kStages) & 1;
-              if (!bar_wait(smem_addr(&ctrl->empty[s]), ph ^ 1, abort)) { ok = false; break; }
+              if (!bar_wait(smem_addr(&ctrl->empty[s]), ph ^ 1, abort, p.limit_ns)) { ok = false; break; }
               const uint32_t bar = smem_addr(&ctrl->full[s]);
               const uint32_t a = stage0 + s * kStageBytes, b = a + kABytes;
               bar_expect_tx(bar, kStageBytes);
@@ -348,14 +351,14 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
         int c0, c1;
         group_chunks(p, (int)(item % p.n_groups), c0, c1);
         for (int c = c0; ok && c < c1; ++c, ++acc_it) {
-          if (!bar_wait(smem_addr(&ctrl->acc_empty[0]), (acc_it & 1) ^ 1, abort)) { ok = false; break; }
+          if (!bar_wait(smem_addr(&ctrl->acc_empty[0]), (acc_it & 1) ^ 1, abort, p.limit_ns)) { ok = false; break; }
           tc_fence_after_sync();
           for (int pass = 0; ok && pass < (NEED_U ? 2 : 1); ++pass) {
             const int nk = pass ? p.kt_blocks : p.ks_blocks;
             const uint32_t tmem_d = tmem_base + (pass ? kBN : 0);
             for (int kb = 0; kb < nk; ++kb, ++it) {
               const uint32_t s = it % kStages, ph = (it / kStages) & 1;
-              if (!bar_wait(smem_addr(&ctrl->full[s]), ph, abort)) { ok = false; break; }
+              if (!bar_wait(smem_addr(&ctrl->full[s]), ph, abort, p.limit_ns)) { ok = false; break; }
               tc_fence_after_sync();
               const uint32_t a = stage0 + s * kStageBytes, b = a + kABytes;
               issue_kblock<false, false>(tmem_d, a, b, kb == 0);
@@ -402,7 +405,7 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
         y = __float_as_int(inf[4]);
       }
       for (int c = c0; ok && c < c1; ++c, ++acc_it) {
-        if (!__all_sync(0xffffffffu, bar_wait(smem_addr(&ctrl->acc_full[0]), acc_it & 1, abort))) {
+        if (!__all_sync(0xffffffffu, bar_wait(smem_addr(&ctrl->acc_full[0]), acc_it & 1, abort, p.limit_ns))) {
           ok = false;   // the same decision in every lane: tcgen05.ld below is warp-collective
           break;
         }
@@ -463,7 +466,8 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
             __nv_bfloat16* gp = p.G + ((int64_t)tile_c * kBM + row) * p.ldG + col;
 #pragma unroll
             for (int v = 0; v < 4; ++v)
-              if (col + v * 8 < p.V)
+              if (col + v * 8 < p.V &&
+                  ADWIN_CHK(tile_c < p.max_tiles && col + v * 8 + 8 <= p.ldG, p.status))
                 *reinterpret_cast<uint4*>(gp + v * 8) =
                     make_uint4(pk[v * 4], pk[v * 4 + 1], pk[v * 4 + 2], pk[v * 4 + 3]);
           }
@@ -471,9 +475,9 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
         tc_fence_before_sync();
         bar_arrive(smem_addr(&ctrl->acc_empty[0]));
       }
-      if (GRAD && ok)
+      if (GRAD && ok && ADWIN_CHK(tile_c < p.max_tiles && g < p.n_groups, p.status))
         p.part[(((int64_t)tile_c * p.n_groups + g) * 2 + half) * kBM + row] = q;
-      if (!GRAD && ok) {
+      if (!GRAD && ok && ADWIN_CHK(tile < p.max_tiles && g < p.n_groups && row < kBM, p.status)) {
         float* o = p.part + ((((int64_t)tile * p.n_groups + g) * 2 + half) * kRecFields) * kBM + row;
         o[0 * kBM] = acc.m2s;
         o[1 * kBM] = acc.S;
@@ -620,6 +624,7 @@ struct GemmParams {
   int64_t ldc;
   int c_is_bf16;
   int32_t* status;
+  uint64_t limit_ns;            // limit of the handshake waits
 };
 
 template <bool A_MN, bool B_MN>
@@ -666,7 +671,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int m0 = (int)(item / p.n_tiles) * kBM, n0 = (int)(item % p.n_tiles) * kBN;
         for (int kb = 0; kb < nk; ++kb, ++it) {
           const uint32_t s = it % kStages, ph = (it / kStages) & 1;
-          if (!bar_wait(smem_addr(&ctrl->empty[s]), ph ^ 1, abort)) { ok = false; break; }
+          if (!bar_wait(smem_addr(&ctrl->empty[s]), ph ^ 1, abort, p.limit_ns)) { ok = false; break; }
           const uint32_t bar = smem_addr(&ctrl->full[s]);
           const uint32_t a = stage0 + s * kStageBytes, b = a + kABytes;
           bar_expect_tx(bar, kStageBytes);
@@ -686,12 +691,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       bool ok = true;
       for (int64_t item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++acc_it) {
         const uint32_t slot = acc_it & 1, aph = (acc_it >> 1) & 1;
-        if (!bar_wait(smem_addr(&ctrl->acc_empty[slot]), aph ^ 1, abort)) { ok = false; break; }
+        if (!bar_wait(smem_addr(&ctrl->acc_empty[slot]), aph ^ 1, abort, p.limit_ns)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t tmem_d = tmem_base + slot * kBN;
         for (int kb = 0; kb < nk; ++kb, ++it) {
           const uint32_t s = it % kStages, ph = (it / kStages) & 1;
-          if (!bar_wait(smem_addr(&ctrl->full[s]), ph, abort)) { ok = false; break; }
+          if (!bar_wait(smem_addr(&ctrl->full[s]), ph, abort, p.limit_ns)) { ok = false; break; }
           tc_fence_after_sync();
           const uint32_t a = stage0 + s * kStageBytes, b = a + kABytes;
           issue_kblock<A_MN, B_MN>(tmem_d, a, b, kb == 0);
@@ -717,14 +722,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const uint32_t slot = acc_it & 1, aph = (acc_it >> 1) & 1;
       const int64_t m = (int64_t)(item / p.n_tiles) * kBM + row;
       const int64_t n0 = (int64_t)(item % p.n_tiles) * kBN + half * 128;
-      if (!__all_sync(0xffffffffu, bar_wait(smem_addr(&ctrl->acc_full[slot]), aph, abort))) {
+      if (!__all_sync(0xffffffffu, bar_wait(smem_addr(&ctrl->acc_full[slot]), aph, abort, p.limit_ns))) {
         ok = false;
         break;
       }
       tc_fence_after_sync();
       int64_t dst = m;
       if (p.row_map) dst = (m < p.M) ? p.row_map[m] : -1;
-      const bool store = m < p.M && dst >= 0;
+      const bool store = m < p.M && dst >= 0 && ADWIN_CHK(n0 >= 0 && n0 < (int64_t)p.n_tiles * kBN, p.status);
       const uint32_t t_lane =
           tmem_base + ((uint32_t)(quad * 32) << 16) + slot * kBN + (uint32_t)(half * 128);
 #pragma unroll 1
@@ -802,6 +807,7 @@ cudaError_t launch_tc_gemm(const void* A, int64_t lda, bool a_mn, const void* B,
   p.ldc = ldc;
   p.c_is_bf16 = c_bf16 ? 1 : 0;
   p.status = status;
+  p.limit_ns = handshake_wait_limit_ns();
   cudaError_t e;
 #define ADWIN_LAUNCH_GEMM(AM, BM_)                                                    \
   do {                                                                                \
@@ -886,6 +892,8 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
   sp.info = info;
   sp.G = G;
   sp.ldG = L.ldG;
+  sp.max_tiles = L.max_tiles;
+  sp.limit_ns = handshake_wait_limit_ns();
   sp.status = status;
   if ((e = opt_in_smem(lm_sweep_kernel<false, true>)) != cudaSuccess) return e;
   lm_sweep_kernel<false, true><<<sm_count, kThreads, kSmemBytes, s>>>(m_hs, m_ws, m_ht, m_wt, sp);

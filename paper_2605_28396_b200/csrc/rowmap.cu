@@ -66,6 +66,7 @@ __global__ void __launch_bounds__(kMapThreads) rowmap_kernel(
     }
     int64_t run = part[tid] - sum;
     for (int64_t b = b0; b < b1; ++b) {
+      if (!ADWIN_CHK(b >= 0 && b < B && run >= 0 && run <= B * T, status)) break;
       offsets[b] = run;
       run += range[b];
     }
@@ -98,7 +99,7 @@ __global__ void __launch_bounds__(kMapThreads) rowmap_kernel(
     int E, P;
     bool bad;
     clamp_lengths(window[b], rollout_len ? rollout_len[b] : (int32_t)T, T, flags, E, P, bad);
-    if (t >= P) {
+    if (t >= P && ADWIN_CHK(b < B && t >= 0 && t < T, status)) {
       kl[i] = 0.f;
       logratio[i] = 0.f;
       if (gsq) gsq[i] = 0.f;

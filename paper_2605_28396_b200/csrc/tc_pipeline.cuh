@@ -98,14 +98,16 @@ __device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile
   if (*abort) return false;
   const uint64_t t0 = timer_ns();
   for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 64; ++i)
-      if (bar_try_wait(bar, parity)) return true;
-    if (*abort) return false;
+    // tested before each batch of polls: a limit shorter than one poll gives up at the first wait
+    // that is not already satisfied
     if (timer_ns() - t0 > limit_ns) {
       *abort = 1;
       return false;
     }
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (bar_try_wait(bar, parity)) return true;
+    if (*abort) return false;
   }
 }
 // The same wait for the give-up path itself: it ignores the abort flag (it runs after the flag is

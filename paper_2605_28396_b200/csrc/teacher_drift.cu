@@ -98,6 +98,7 @@ __global__ void __launch_bounds__(kDriftThreads) teacher_drift_kernel(
       int64_t i = tid;
       for (; i + (kDriftUnroll - 1) * kDriftThreads < pieces; i += kDriftUnroll * kDriftThreads) {
         uint4 v[kDriftUnroll];
+        if (!ADWIN_CHK((i + (kDriftUnroll - 1) * kDriftThreads + 1) * N <= ld, status)) break;
 #pragma unroll
         for (int k = 0; k < kDriftUnroll; ++k) v[k] = __ldcs(src + i + k * kDriftThreads);
 #pragma unroll
@@ -109,11 +110,13 @@ __global__ void __launch_bounds__(kDriftThreads) teacher_drift_kernel(
       }
       for (; i < pieces; i += kDriftThreads) {
         float u[Elem<TIn>::N];
+        if (!ADWIN_CHK((i + 1) * N <= ld, status)) break;
         Elem<TIn>::unpack(__ldcs(src + i), u);
         drift_piece<Elem<TIn>::N>(u, uy, a);
       }
     } else {
       for (int64_t i = tid; i < pieces; i += kDriftThreads) {
+        if (!ADWIN_CHK(i < ld, status)) break;
         float u[1] = {Elem<TIn>::load1(urow, i)};
         drift_piece<1>(u, uy, a);
       }

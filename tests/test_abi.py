@@ -32,6 +32,42 @@ def test_every_declared_symbol_is_exported(L):
     assert set(api.EXPORTS) <= set(names)
 
 
+def test_checked_flavour_builds_and_exports_the_same_symbols():
+    lib = ctypes.CDLL(str(build.build(checked=True)))
+    for n in declared_functions():
+        assert hasattr(lib, n), f"{n} missing from the bounds-checked flavour"
+    lib.adwin_version.restype = ctypes.c_int
+    assert lib.adwin_version() == api.lib().adwin_version()
+
+
+def test_lmhead_entry_point_rejects_bad_arguments_on_the_host(L):
+    fake = ctypes.c_void_p(4096)   # never dereferenced: validation fails first
+    status = ctypes.c_void_p(8192)
+
+    def call(**over):
+        a = dict(hs=fake, ws=fake, ht=fake, wt=fake, B=2, T=16, V=256, ds=64, dt=64, tok=fake,
+                 win=fake, roll=None, scale=1.0, mode=0, flags=0, gh=None, ghd=0, gw=None, kl=fake,
+                 c=fake, gsq=None, ls=None, lt=None, max_rows=0, ws_=fake, wsb=1 << 30, st=status)
+        a.update(over)
+        return L.adwin_opd_kl_lmhead_fwd_bwd(a["hs"], a["ws"], a["ht"], a["wt"], a["B"], a["T"],
+                                             a["V"], a["ds"], a["dt"], a["tok"], a["win"],
+                                             a["roll"], a["scale"], a["mode"], a["flags"], a["gh"],
+                                             a["ghd"], a["gw"], a["kl"], a["c"], a["gsq"], a["ls"],
+                                             a["lt"], a["max_rows"], a["ws_"], a["wsb"], a["st"],
+                                             None)
+    assert call(mode=7) == 4 and call(flags=4) == 4            # ADWIN_ERR_DTYPE
+    assert call(V=0) == 2 and call(ds=0) == 2 and call(B=-1) == 2
+    assert call(st=None) == 1 and call(kl=None) == 1 and call(ws=None) == 1
+    assert call(V=260) == 8 and call(dt=68) == 8               # not multiples of 8
+    assert call(hs=ctypes.c_void_p(4100)) == 3                 # misaligned
+    assert call(wsb=1024) == 6 and call(ws_=None) == 6         # workspace
+    assert call(B=0) == 0                                      # empty batch: nothing to do
+    need = api.adwin_lmhead_workspace_bytes(2, 16, 256, 64, 64)
+    assert need > 0 and need % 1024 == 0
+    assert api.adwin_lmhead_workspace_bytes(16, 4096, 151936, 2048, 2560, 36000) < \
+        api.adwin_lmhead_workspace_bytes(16, 4096, 151936, 2048, 2560, 0)
+
+
 def test_version_and_status_strings(L):
     assert L.adwin_version() >= 1
     assert L.adwin_status_string(0) == b"ADWIN_OK"

@@ -330,3 +330,28 @@ def test_window_reduce_is_the_brute_force_prefix_sum():
         assert seq[b, 3] == E
     np.testing.assert_allclose(batch, seq.sum(0), rtol=1e-14)
     assert (seq[0] == 0).all()
+
+
+def test_gsq_term_scale_bounds_the_terms_of_the_one_sweep_form():
+    # the scale must dominate each of the three sums the expanded form combines, and the expanded
+    # form must equal gsq; with the peak as the sample the scale stays near gsq, off the peak it
+    # grows like 1/(1-p_max)^2
+    V = 300
+    z = RNG.normal(0, 1, V)
+    z[7] += 12.0                                   # a peaked row: p_7 ~ 0.99
+    u = z + RNG.normal(0, 2, V)
+    for y, lo, hi in ((7, 1.0, 20.0), (11, 50.0, 1e9)):
+        r = O.row(z, u, y)
+        p = np.exp(z - r["lse_s"])
+        d = (z - u) - (z[y] - u[y])
+        c0 = float(np.sum(p * (z - u))) - (z[y] - u[y])
+        B2, B1, B0 = np.sum(p * p * d * d), np.sum(p * p * d), np.sum(p * p)
+        assert B2 - 2 * c0 * B1 + c0 * c0 * B0 == pytest.approx(r["gsq"], rel=1e-9)
+        sc = O.row_gsq_term_scale(z, u, y)
+        assert sc >= max(B2, abs(2 * c0 * B1), c0 * c0 * B0) * (1 - 1e-12)
+        assert sc == pytest.approx(2 * (B2 + c0 * c0 * B0), rel=1e-12)
+        assert lo <= sc / r["gsq"] <= hi
+    s = O.row(z, u, 11, alpha=0.5, mode=O.MODE_SAMPLED)
+    p11 = np.exp(z[11] - s["lse_s"])
+    want = (0.5 * s["c"]) ** 2 * (np.sum(p * p) + p11 ** 2 + (1 - p11) ** 2)
+    assert O.row_gsq_term_scale(z, u, 11, 0.5, O.MODE_SAMPLED) == pytest.approx(want, rel=1e-12)
