@@ -89,9 +89,9 @@ int adwin_version(void);
  * for its own copies and MMAs in flight (those waits keep the full limit), frees its tensor
  * memory and returns; the outputs of that call are invalid, the context stays usable.  This sets
  * the limit of those handshake waits for the launches that follow, process-wide, in nanoseconds
- * (default 2 s; 0 restores the default).  A limit of a few nanoseconds makes the first wait that
- * is not already satisfied run out, which is how the tests exercise the give-up path; there is
- * no other use for it.  The paper has no counterpart.
+ * (default 2 s; 0 restores the default).  A limit below 16 ns makes every wait that is not
+ * satisfied at the moment it is reached run out, which is how the tests exercise the give-up path; there
+ * is no other use for it.  The paper has no counterpart.
  */
 void adwin_diag_set_wait_limit_ns(uint64_t ns);
 

@@ -131,6 +131,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Non-blocking test of a phase (try_wait may suspend the thread for a while before it answers).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -206,12 +218,15 @@ __device__ __forceinline__ uint64_t global_timer() {
 template <bool CLUSTER>
 __device__ __forceinline__ bool bounded_wait_lane(uint32_t bar, uint32_t parity,
                                                   volatile int* abort, uint64_t limit_ns) {
+  if (limit_ns < 16) {   // diagnostic setting: a wait that is not satisfied right now runs out
+    if (mbar_test_wait(bar, parity)) return true;
+    *abort = 1;
+    return false;
+  }
   if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
   if (*abort) return false;
   const uint64_t t0 = global_timer();
   for (;;) {
-    // the limit is tested before each batch of polls, so that a limit shorter than one poll gives
-    // up at the first wait that is not already satisfied
     if (global_timer() - t0 > limit_ns) {
       *abort = 1;
       return false;

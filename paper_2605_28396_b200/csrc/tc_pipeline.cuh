@@ -89,17 +89,32 @@ __device__ __forceinline__ bool bar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Non-blocking test of a phase (try_wait may suspend the thread for a while before it answers).
+__device__ __forceinline__ bool bar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // Wait for the phase with the given parity to complete.  Returns false when the CTA has given up
 // (another role ran out of time) or when this wait itself exceeds the limit, in which case it
 // raises the CTA's abort flag.
 __device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile int* abort,
                                          uint64_t limit_ns = kWaitLimitNs) {
+  if (limit_ns < 16) {   // diagnostic setting: a wait that is not satisfied right now runs out
+    if (bar_test_wait(bar, parity)) return true;
+    *abort = 1;
+    return false;
+  }
   if (bar_try_wait(bar, parity)) return true;
   if (*abort) return false;
   const uint64_t t0 = timer_ns();
   for (;;) {
-    // tested before each batch of polls: a limit shorter than one poll gives up at the first wait
-    // that is not already satisfied
     if (timer_ns() - t0 > limit_ns) {
       *abort = 1;
       return false;
