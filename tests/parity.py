@@ -54,7 +54,8 @@ def oracle_batch(batch, rows=None, **kw):
 GSQ_SCALE_ULPS = 64
 
 
-def check_scalars(got, ref, rtol, processed_mask, name="", grad_mask=None, gsq_scale=None):
+def check_scalars(got, ref, rtol, processed_mask, name="", grad_mask=None, gsq_scale=None,
+                  rtol_gsq_grad=None):
     """got: namespace of device tensors; ref: oracle dict; mask: [B,T] bool of processed rows;
     grad_mask: rows whose gradient was written (their gsq is summed from the gradient);
     gsq_scale: oracle's term scale of the one-sweep gsq, for the rows outside grad_mask."""
@@ -77,7 +78,7 @@ def check_scalars(got, ref, rtol, processed_mask, name="", grad_mask=None, gsq_s
         err = np.abs(q - b)[valid]
         rq = np.full(b.shape, RTOL_GSQ_SINGLE_SWEEP)
         if grad_mask is not None:
-            rq[grad_mask] = RTOL_GSQ
+            rq[grad_mask] = RTOL_GSQ if rtol_gsq_grad is None else rtol_gsq_grad
         lim_all = rq * np.abs(b) + 1e-30
         if gsq_scale is not None:
             extra = GSQ_SCALE_ULPS * 2.0 ** -23 * np.asarray(gsq_scale)
