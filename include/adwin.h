@@ -293,6 +293,44 @@ int adwin_opd_kl_lmhead_fwd_bwd(const void* hidden_student, const void* w_studen
                                 size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
 
 /*
+ * Prefix-versus-full alignment audit (Section 4.2) in the space of the student's LM-head weight,
+ * on a returned probe batch given as hidden states.  For every candidate length L_j the prefix
+ * gradient is dW^(L_j) = sum_b sum_{t < min(L_j, R_b)} G[b,t,:]^T h_s[b,t,:] and the full-horizon
+ * reference dW^full the same sum over t < R_b (G = the logit gradient of the selected estimator,
+ * every position of every rollout); then
+ *   rho_w(L_j) = <dW^(L_j), dW^full> / (|dW^(L_j)| |dW^full|)     (the cosine after batch aggregation),
+ * SNR = rho^2 / (1 - rho^2), admissible <=> rho_w >= rho_star, *L_next = the shortest admissible
+ * candidate (the scheduler rule), or the largest one with ADWIN_ALIGN_NONE_ADMISSIBLE.  Unlike the
+ * logit-space audit of adwin_probe_align this cosine sees the cancellation between positions and
+ * samples (Figure 5) and can be negative.  A zero full norm gives rho = 1 and ADWIN_ALIGN_DEGENERATE,
+ * a zero prefix norm rho = 0.
+ *
+ * hidden_*, w_*, tokens, rollout_len (NULL = T), grad_mode, max_rows (bound on sum_b R_b; <= 0 =
+ * B*T), dev_status: as in adwin_opd_kl_lmhead_fwd_bwd.
+ * candidates_host : HOST pointer to K strictly ascending multiples of 64 (they cut the positions
+ *                   into bins of whole 64-row blocks), 1 <= K <= 16; NULL selects the paper's list
+ *                   {64,...,2048} (then K must be 0 or 6).  rho_star <= 0 selects sqrt(2)/2.
+ * kl, logratio, gsq : [B,T] fp32 per-token outputs over t < R_b (kl, logratio required).
+ * batch_stats [K,4] = { rho_w, snr, admissible (0/1), n_tokens } float64; L_next, flags_out int32:
+ *                   device pointers.
+ * workspace       : >= adwin_lmhead_align_workspace_bytes(...) bytes, 1024-byte aligned: the
+ *                   workspace of the fused pass plus K+1 fp32 matrices of the size of W_s.
+ * The products run in bf16 with fp32 accumulation, G rounded to bf16 once; the cosines are formed
+ * in float64 from the fp32 bin matrices in a fixed order.
+ */
+size_t adwin_lmhead_align_workspace_bytes(int64_t B, int64_t T, int64_t V, int64_t d_s,
+                                          int64_t d_t, int64_t max_rows, int32_t K);
+int adwin_lmhead_weight_align(const void* hidden_student, const void* w_student,
+                              const void* hidden_teacher, const void* w_teacher, int64_t B,
+                              int64_t T, int64_t V, int64_t d_s, int64_t d_t,
+                              const int32_t* tokens, const int32_t* rollout_len,
+                              const int32_t* candidates_host, int32_t K, double rho_star,
+                              int grad_mode, float* kl, float* logratio, float* gsq,
+                              double* batch_stats, int32_t* L_next, int32_t* flags_out,
+                              int64_t max_rows, void* workspace, size_t workspace_bytes,
+                              int32_t* dev_status, void* cuda_stream);
+
+/*
  * The same pass for logits that live in HOST memory (pinned memory gives asynchronous copies).
  * Only the rows inside the processed range cross PCIe -- the window skip of Section 4.1 saves the
  * transfer as well as the arithmetic -- in stages of at most rows_per_stage rows of one sequence;

@@ -30,7 +30,8 @@ EXPORTS = ("adwin_version", "adwin_status_string", "adwin_workspace_bytes",
            "adwin_no_alloc_max_sequences", "adwin_opd_kl_fwd_bwd_no_alloc",
            "adwin_return_to_go", "adwin_opd_kl_fwd_bwd_weighted", "adwin_teacher_drift",
            "adwin_drift_curves", "adwin_lmhead_workspace_bytes", "adwin_opd_kl_lmhead_fwd_bwd",
-           "adwin_diag_set_wait_limit_ns")
+           "adwin_diag_set_wait_limit_ns", "adwin_lmhead_align_workspace_bytes",
+           "adwin_lmhead_weight_align")
 
 _lib = None
 
@@ -105,6 +106,12 @@ def lib():
                                                   vp, f32, ctypes.c_int, ctypes.c_int, vp,
                                                   ctypes.c_int, vp, vp, vp, vp, vp, vp, i64, vp,
                                                   sz, vp, vp]
+        L.adwin_lmhead_align_workspace_bytes.restype = sz
+        L.adwin_lmhead_align_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, i64, i32]
+        L.adwin_lmhead_weight_align.restype = ctypes.c_int
+        L.adwin_lmhead_weight_align.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, i64, vp, vp,
+                                                vp, i32, f64, ctypes.c_int, vp, vp, vp, vp, vp,
+                                                vp, i64, vp, sz, vp, vp]
         L.adwin_diag_set_wait_limit_ns.restype = None
         L.adwin_diag_set_wait_limit_ns.argtypes = [ctypes.c_uint64]
         _lib = L
@@ -428,3 +435,44 @@ def adwin_opd_kl_lmhead_fwd_bwd(hidden_student, w_student, hidden_teacher, w_tea
 def adwin_diag_set_wait_limit_ns(ns: int) -> None:
     """Diagnostic: limit of the kernels' handshake waits for the launches that follow (0 = default)."""
     lib().adwin_diag_set_wait_limit_ns(int(ns))
+
+
+def adwin_lmhead_weight_align(hidden_student, w_student, hidden_teacher, w_teacher, tokens,
+                              rollout_len=None, candidates=None, rho_star=0.0, *,
+                              grad_mode=GRAD_FULL_KL, max_rows=0, workspace=None, dev_status=None):
+    """Section 4.2's prefix/full cosine in the space of the student's LM-head weight (adwin.h).
+
+    candidates: a host sequence of ascending multiples of 64, or None for the paper's list.
+    Returns a namespace with batch_stats [K,4] (rho_w, snr, admissible, n_tokens), L_next, flags,
+    kl, logratio, gsq, dev_status, candidates.
+    """
+    B, T, ds = hidden_student.shape
+    V = w_student.shape[0]
+    dt = hidden_teacher.shape[2]
+    dev = hidden_student.device
+    for t in (hidden_student, w_student, hidden_teacher, w_teacher):
+        if t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise TypeError("hidden states and LM heads must be contiguous bf16 tensors")
+    cands = list(DEFAULT_CANDIDATES) if candidates is None else [int(x) for x in candidates]
+    K = len(cands)
+    carr = (ctypes.c_int32 * max(K, 1))(*cands)
+    kl = torch.empty((B, T), dtype=torch.float32, device=dev)
+    logratio = torch.empty((B, T), dtype=torch.float32, device=dev)
+    gsq = torch.empty((B, T), dtype=torch.float32, device=dev)
+    stats = torch.empty((K, 4), dtype=torch.float64, device=dev)
+    L_next = torch.zeros(1, dtype=torch.int32, device=dev)
+    flags = torch.zeros(1, dtype=torch.int32, device=dev)
+    need = int(lib().adwin_lmhead_align_workspace_bytes(B, T, V, ds, dt, int(max_rows), K))
+    if workspace is None:
+        workspace = torch.empty(need + 1024, dtype=torch.uint8, device=dev)
+    off = (-workspace.data_ptr()) % 1024
+    if dev_status is None:
+        dev_status = torch.zeros(1, dtype=torch.int32, device=dev)
+    _check(lib().adwin_lmhead_weight_align(
+        _ptr(hidden_student), _ptr(w_student), _ptr(hidden_teacher), _ptr(w_teacher), B, T, V, ds,
+        dt, _ptr(tokens), _ptr(rollout_len), ctypes.cast(carr, ctypes.c_void_p), K,
+        float(rho_star), int(grad_mode), _ptr(kl), _ptr(logratio), _ptr(gsq), _ptr(stats),
+        _ptr(L_next), _ptr(flags), int(max_rows), ctypes.c_void_p(workspace.data_ptr() + off),
+        workspace.numel() - off, _ptr(dev_status), _stream(dev)))
+    return SimpleNamespace(batch_stats=stats, L_next=L_next, flags=flags, kl=kl, logratio=logratio,
+                           gsq=gsq, dev_status=dev_status, candidates=cands, workspace=workspace)

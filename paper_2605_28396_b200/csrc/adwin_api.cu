@@ -377,7 +377,69 @@ int adwin_opd_kl_lmhead_fwd_bwd(const void* hidden_student, const void* w_studen
   return ADWIN_OK;
 }
 
+size_t adwin_lmhead_align_workspace_bytes(int64_t B, int64_t T, int64_t V, int64_t d_s,
+                                          int64_t d_t, int64_t max_rows, int32_t K) {
+  if (B < 0) B = 0;
+  if (T < 0) T = 0;
+  if (V < 1) V = 1;
+  if (d_s < 1) d_s = 1;
+  if (d_t < 1) d_t = 1;
+  if (K < 1) K = 6;
+  if (K > 16) K = 16;
+  return lmhead_align_workspace_bytes(B, T, V, d_s, d_t, max_rows, K);
+}
+
+int adwin_lmhead_weight_align(const void* hidden_student, const void* w_student,
+                              const void* hidden_teacher, const void* w_teacher, int64_t B,
+                              int64_t T, int64_t V, int64_t d_s, int64_t d_t,
+                              const int32_t* tokens, const int32_t* rollout_len,
+                              const int32_t* candidates_host, int32_t K, double rho_star,
+                              int grad_mode, float* kl, float* logratio, float* gsq,
+                              double* batch_stats, int32_t* L_next, int32_t* flags_out,
+                              int64_t max_rows, void* workspace, size_t workspace_bytes,
+                              int32_t* dev_status, void* cuda_stream) {
+  static const int32_t kPaperList[6] = {64, 128, 256, 512, 1024, 2048};
+  if (grad_mode != ADWIN_GRAD_FULL_KL && grad_mode != ADWIN_GRAD_SAMPLED) return ADWIN_ERR_DTYPE;
+  if (!candidates_host) {
+    if (K != 0 && K != 6) return ADWIN_ERR_SHAPE;
+    candidates_host = kPaperList;
+    K = 6;
+  }
+  if (K < 1 || K > 16) return ADWIN_ERR_SHAPE;
+  for (int i = 0; i < K; ++i) {
+    if (candidates_host[i] <= 0 || candidates_host[i] % 64 != 0) return ADWIN_ERR_SHAPE;
+    if (i > 0 && candidates_host[i] <= candidates_host[i - 1]) return ADWIN_ERR_SHAPE;
+  }
+  if (B < 0 || T < 0 || B > 65536 || T > kMaxT || V < 1 || V > kMaxV || d_s < 1 || d_t < 1 ||
+      d_s > (int64_t(1) << 20) || d_t > (int64_t(1) << 20))
+    return ADWIN_ERR_SHAPE;
+  if (!dev_status || !batch_stats || !L_next || !flags_out) return ADWIN_ERR_NULL;
+  if (B > 0 && T > 0 &&
+      (!hidden_student || !w_student || !hidden_teacher || !w_teacher || !tokens || !kl || !logratio))
+    return ADWIN_ERR_NULL;
+  if ((V % 8) || (d_s % 8) || (d_t % 8) || B * T > (int64_t(1) << 30)) return ADWIN_ERR_UNSUPPORTED;
+  if (!aligned(hidden_student, 16) || !aligned(w_student, 16) || !aligned(hidden_teacher, 16) ||
+      !aligned(w_teacher, 16) || !aligned(tokens, 4) || !aligned(rollout_len, 4) ||
+      !aligned(kl, 4) || !aligned(logratio, 4) || !aligned(gsq, 4) || !aligned(batch_stats, 8) ||
+      !aligned(L_next, 4) || !aligned(flags_out, 4) || !aligned(dev_status, 4))
+    return ADWIN_ERR_ALIGN;
+  if (!workspace || !aligned(workspace, 1024) ||
+      workspace_bytes < lmhead_align_workspace_bytes(B, T, V, d_s, d_t, max_rows, K))
+    return ADWIN_ERR_WORKSPACE;
+  if (!(rho_star > 0.0)) rho_star = 0.70710678118654752440;  // sqrt(2)/2
+  const int sms = sm_count_of_current_device();
+  if (sms <= 0) return ADWIN_ERR_CUDA;
+  if (launch_lmhead_weight_align(hidden_student, w_student, hidden_teacher, w_teacher, B, T, V, d_s,
+                                 d_t, tokens, rollout_len, candidates_host, K, rho_star, grad_mode,
+                                 kl, logratio, gsq, batch_stats, L_next, flags_out, workspace,
+                                 max_rows, dev_status, sms,
+                                 static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return ADWIN_ERR_CUDA;
+  return ADWIN_OK;
+}
+
 #ifdef ADWIN_DEV_EXPORTS
+void adwin_dev_set_sweep_bn(int bn) { set_sweep_tile_columns(bn); }
 // Development build only: the tensor-core GEMM on its own, C = A B (bf16 in, fp32 or bf16 out).
 int adwin_dev_gemm(const void* A, int64_t lda, int a_mn, const void* Bm, int64_t ldb, int b_mn,
                    int64_t M, int64_t N, int64_t K, void* C, int64_t ldc, int c_bf16,

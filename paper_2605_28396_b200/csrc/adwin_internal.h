@@ -65,6 +65,7 @@ cudaError_t launch_drift_curves(const float* entropy, const int32_t* rank,
                                 double* bf_mean, int32_t* n_active, cudaStream_t s);
 
 // Fused LM-head form (lmhead.cu).
+void set_sweep_tile_columns(int bn);
 size_t lmhead_workspace_bytes(int64_t B, int64_t T, int64_t V, int64_t ds, int64_t dt,
                               int64_t max_rows, bool want_grad, bool range_full);
 cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const void* wt, int64_t B,
@@ -72,10 +73,22 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
                           const int32_t* window, const int32_t* rollout_len, float alpha, int mode,
                           int flags, void* dH, int dh_dtype, float* dW, float* kl, float* logratio,
                           float* gsq, float* lse_s, float* lse_t, void* workspace,
-                          int64_t max_rows, int32_t* status, int sm_count, cudaStream_t s);
+                          int64_t max_rows, int32_t* status, int sm_count, cudaStream_t s,
+                          bool keep_G = false);
+size_t lmhead_align_workspace_bytes(int64_t B, int64_t T, int64_t V, int64_t ds, int64_t dt,
+                                    int64_t max_rows, int K);
+cudaError_t launch_lmhead_weight_align(const void* hs, const void* ws, const void* ht,
+                                       const void* wt, int64_t B, int64_t T, int64_t V, int64_t ds,
+                                       int64_t dt, const int32_t* tokens,
+                                       const int32_t* rollout_len, const int32_t* cand_host, int K,
+                                       double rho_star, int mode, float* kl, float* logratio,
+                                       float* gsq, double* batch_stats, int32_t* L_next,
+                                       int32_t* flags_out, void* workspace, int64_t max_rows,
+                                       int32_t* status, int sm_count, cudaStream_t s);
 cudaError_t launch_tc_gemm(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
                            bool b_mn, int64_t M, int64_t N, int64_t K, void* C, int64_t ldc,
                            bool c_bf16, const int32_t* m_tiles_dev, const int32_t* k_tiles_dev,
-                           const int32_t* row_map, int32_t* status, int sm_count, cudaStream_t s);
+                           const int32_t* row_map, int32_t* status, int sm_count, cudaStream_t s,
+                           const int32_t* k_list = nullptr, const int32_t* k_count_dev = nullptr);
 
 }  // namespace adwin

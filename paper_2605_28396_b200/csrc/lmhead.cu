@@ -273,13 +273,23 @@ __device__ __forceinline__ void group_chunks(const SweepParams& p, int g, int& c
   if (c0 > c1) c0 = c1;
 }
 
+// MOMENTS = false drops the squared-norm moments from sweep 1 (when every processed row gets its
+// gsq from sweep 2, or no gsq is asked for).
 // GRAD = false: sweep 1 (statistics).  GRAD = true: sweep 2 (logit gradient); NEED_U = false
 // skips the teacher product there (the sampled-token estimator of Eq. 4 does not need it).
-template <bool GRAD, bool NEED_U>
+template <bool GRAD, bool NEED_U, int BN, bool MOMENTS = true>
 __global__ void __launch_bounds__(kThreads, 1)
 lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constant__ CUtensorMap map_ws,
                 const __grid_constant__ CUtensorMap map_ht, const __grid_constant__ CUtensorMap map_wt,
                 const SweepParams p) {
+  // BN = 256: one accumulator pair (student + teacher tile) fills the 512 TMEM columns, the
+  // epilogue and the MMAs of the next chunk alternate.  BN = 128: two pairs, so the epilogue of a
+  // chunk overlaps the MMAs of the next, at 1.5x the operand bytes per flop.
+  constexpr int kSt = BN == 256 ? 4 : 6;            // pipeline stages
+  constexpr int kStB = kABytes + BN * kBK * 2;      // bytes per stage
+  constexpr int kAcc = kTmemCols / (2 * BN);        // accumulator pairs
+  constexpr int kHalf = BN / 2;                     // columns per epilogue warpgroup
+  static_assert(kSt <= kMaxStages && kSt * kStB <= kStages * kStageBytes, "stage budget");
   extern __shared__ uint8_t smem_raw[];
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem_raw);
   const uint32_t stage0 = (smem_addr(smem_raw) + kCtrlBytes + 1023u) & ~1023u;
@@ -287,12 +297,14 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
   volatile int* abort = &ctrl->abort;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < kSt; ++s) {
       bar_init(smem_addr(&ctrl->full[s]), 1);
       bar_init(smem_addr(&ctrl->empty[s]), 1);
     }
-    bar_init(smem_addr(&ctrl->acc_full[0]), 1);
-    bar_init(smem_addr(&ctrl->acc_empty[0]), kEpiThreads);
+    for (int s = 0; s < kAcc; ++s) {
+      bar_init(smem_addr(&ctrl->acc_full[s]), 1);
+      bar_init(smem_addr(&ctrl->acc_empty[s]), kEpiThreads);
+    }
     bar_init(smem_addr(&ctrl->drain), 1);
     ctrl->abort = 0;
     bar_init_fence();
@@ -325,21 +337,21 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
             const CUtensorMap* mb = pass ? &map_wt : &map_ws;
             const int nk = pass ? p.kt_blocks : p.ks_blocks;
             for (int kb = 0; kb < nk; ++kb, ++it) {
-              const uint32_t s = it % kStages, ph = (it / kStages) & 1;
+              const uint32_t s = it % kSt, ph = (it / kSt) & 1;
               if (!bar_wait(smem_addr(&ctrl->empty[s]), ph ^ 1, abort, p.limit_ns)) { ok = false; break; }
               const uint32_t bar = smem_addr(&ctrl->full[s]);
-              const uint32_t a = stage0 + s * kStageBytes, b = a + kABytes;
-              bar_expect_tx(bar, kStageBytes);
+              const uint32_t a = stage0 + s * kStB, b = a + kABytes;
+              bar_expect_tx(bar, kStB);
               tma_load_2d(a, ma, kb * kBK, row0, bar);
-              tma_load_2d(b, mb, kb * kBK, c * kBN, bar);
+              tma_load_2d(b, mb, kb * kBK, c * BN, bar);
             }
           }
         }
       }
       if (!ok) {   // give up: let the copies in flight land before the CTA's shared memory goes
-        const uint32_t n_out = it < (uint32_t)kStages ? it : (uint32_t)kStages;
+        const uint32_t n_out = it < (uint32_t)kSt ? it : (uint32_t)kSt;
         for (uint32_t j = it - n_out; j < it; ++j)
-          bar_wait_drain(smem_addr(&ctrl->full[j % kStages]), (j / kStages) & 1);
+          bar_wait_drain(smem_addr(&ctrl->full[j % kSt]), (j / kSt) & 1);
       }
     }
   } else if (warp == 1) {
@@ -351,21 +363,22 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
         int c0, c1;
         group_chunks(p, (int)(item % p.n_groups), c0, c1);
         for (int c = c0; ok && c < c1; ++c, ++acc_it) {
-          if (!bar_wait(smem_addr(&ctrl->acc_empty[0]), (acc_it & 1) ^ 1, abort, p.limit_ns)) { ok = false; break; }
+          const uint32_t slot = acc_it % kAcc, aph = (acc_it / kAcc) & 1;
+          if (!bar_wait(smem_addr(&ctrl->acc_empty[slot]), aph ^ 1, abort, p.limit_ns)) { ok = false; break; }
           tc_fence_after_sync();
           for (int pass = 0; ok && pass < (NEED_U ? 2 : 1); ++pass) {
             const int nk = pass ? p.kt_blocks : p.ks_blocks;
-            const uint32_t tmem_d = tmem_base + (pass ? kBN : 0);
+            const uint32_t tmem_d = tmem_base + slot * (2 * BN) + (pass ? BN : 0);
             for (int kb = 0; kb < nk; ++kb, ++it) {
-              const uint32_t s = it % kStages, ph = (it / kStages) & 1;
+              const uint32_t s = it % kSt, ph = (it / kSt) & 1;
               if (!bar_wait(smem_addr(&ctrl->full[s]), ph, abort, p.limit_ns)) { ok = false; break; }
               tc_fence_after_sync();
-              const uint32_t a = stage0 + s * kStageBytes, b = a + kABytes;
-              issue_kblock<false, false>(tmem_d, a, b, kb == 0);
+              const uint32_t a = stage0 + s * kStB, b = a + kABytes;
+              issue_kblock<false, false, BN>(tmem_d, a, b, kb == 0);
               umma_commit(smem_addr(&ctrl->empty[s]));
             }
           }
-          if (ok) umma_commit(smem_addr(&ctrl->acc_full[0]));
+          if (ok) umma_commit(smem_addr(&ctrl->acc_full[slot]));
         }
       }
       if (!ok) {   // give up: wait until the MMAs already issued have retired
@@ -379,7 +392,7 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
     const int quad = warp & 3;               // TMEM lanes 32*quad .. 32*quad+31
     const int half = ew >> 2;                // columns half*128 .. half*128+127 of the tile
     const int row = quad * 32 + lane;
-    const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * 128);
+    const uint32_t t_quad = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * kHalf);
     uint32_t acc_it = 0;
     bool ok = true;
     for (int64_t item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
@@ -405,18 +418,20 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
         y = __float_as_int(inf[4]);
       }
       for (int c = c0; ok && c < c1; ++c, ++acc_it) {
-        if (!__all_sync(0xffffffffu, bar_wait(smem_addr(&ctrl->acc_full[0]), acc_it & 1, abort, p.limit_ns))) {
+        const uint32_t slot = acc_it % kAcc, aph = (acc_it / kAcc) & 1;
+        const uint32_t t_lane = t_quad + slot * (2 * BN);
+        if (!__all_sync(0xffffffffu, bar_wait(smem_addr(&ctrl->acc_full[slot]), aph, abort, p.limit_ns))) {
           ok = false;   // the same decision in every lane: tcgen05.ld below is warp-collective
           break;
         }
         tc_fence_after_sync();
-        const int64_t col_base = (int64_t)c * kBN + half * 128;
-        const bool ragged = col_base + 128 > p.V;
+        const int64_t col_base = (int64_t)c * BN + half * kHalf;
+        const bool ragged = col_base + kHalf > p.V;
 #pragma unroll 1
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < kHalf / 32; ++j) {
           uint32_t zr[32], ur[32];
           tmem_ld32(t_lane + j * 32, zr);
-          if (NEED_U) tmem_ld32(t_lane + kBN + j * 32, ur);
+          if (NEED_U) tmem_ld32(t_lane + BN + j * 32, ur);
           tmem_ld_wait();
           const int64_t col = col_base + j * 32;
           float z[32], u[32];
@@ -434,7 +449,7 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
               }
           }
           if (!GRAD) {
-            acc_piece<32, true>(z, u, dref, acc);
+            acc_piece<32, MOMENTS>(z, u, dref, acc);
           } else {
             uint32_t pk[16];
 #pragma unroll
@@ -473,7 +488,7 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
           }
         }
         tc_fence_before_sync();
-        bar_arrive(smem_addr(&ctrl->acc_empty[0]));
+        bar_arrive(smem_addr(&ctrl->acc_empty[slot]));
       }
       if (GRAD && ok && ADWIN_CHK(tile_c < p.max_tiles && g < p.n_groups, p.status))
         p.part[(((int64_t)tile_c * p.n_groups + g) * 2 + half) * kBM + row] = q;
@@ -619,6 +634,8 @@ struct GemmParams {
   int m_tiles, n_tiles, k_blocks;
   const int32_t* m_tiles_dev;   // optional device-side override of m_tiles (index into hdr)
   const int32_t* k_tiles_dev;   // optional: k_blocks = 2 * (*k_tiles_dev) (128 rows per tile)
+  const int32_t* k_list;        // optional: contraction row of every k-block (instead of kb*64)
+  const int32_t* k_count_dev;   // with k_list: number of k-blocks
   const int32_t* row_map;       // optional: destination row of every C row, or -1 (skip)
   void* C;
   int64_t ldc;
@@ -660,7 +677,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const uint32_t tmem_base = ctrl->tmem_base;
 
   const int m_tiles = p.m_tiles_dev ? *p.m_tiles_dev : p.m_tiles;
-  const int nk = p.k_tiles_dev ? 2 * (*p.k_tiles_dev) : p.k_blocks;
+  const int nk = p.k_list ? *p.k_count_dev : (p.k_tiles_dev ? 2 * (*p.k_tiles_dev) : p.k_blocks);
   const int64_t n_items = (int64_t)m_tiles * p.n_tiles;
 
   if (warp == 0) {
@@ -675,8 +692,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const uint32_t bar = smem_addr(&ctrl->full[s]);
           const uint32_t a = stage0 + s * kStageBytes, b = a + kABytes;
           bar_expect_tx(bar, kStageBytes);
-          load_operand<A_MN, kBM>(a, &map_a, m0, kb * kBK, bar);
-          load_operand<B_MN, kBN>(b, &map_b, n0, kb * kBK, bar);
+          const int k0 = p.k_list ? p.k_list[kb] : kb * kBK;
+          load_operand<A_MN, kBM>(a, &map_a, m0, k0, bar);
+          load_operand<B_MN, kBN>(b, &map_b, n0, k0, bar);
         }
       }
       if (!ok) {
@@ -789,7 +807,8 @@ cudaError_t opt_in_smem(K kernel) {
 cudaError_t launch_tc_gemm(const void* A, int64_t lda, bool a_mn, const void* B, int64_t ldb,
                            bool b_mn, int64_t M, int64_t N, int64_t K, void* C, int64_t ldc,
                            bool c_bf16, const int32_t* m_tiles_dev, const int32_t* k_tiles_dev,
-                           const int32_t* row_map, int32_t* status, int sm_count, cudaStream_t s) {
+                           const int32_t* row_map, int32_t* status, int sm_count, cudaStream_t s,
+                           const int32_t* k_list, const int32_t* k_count_dev) {
   CUtensorMap ma, mb;
   const bool oka = a_mn ? make_map(&ma, A, M, K, lda, 64) : make_map(&ma, A, K, M, lda, kBM);
   const bool okb = b_mn ? make_map(&mb, B, N, K, ldb, 64) : make_map(&mb, B, K, N, ldb, kBN);
@@ -802,6 +821,8 @@ cudaError_t launch_tc_gemm(const void* A, int64_t lda, bool a_mn, const void* B,
   p.k_blocks = (int)((K + kBK - 1) / kBK);
   p.m_tiles_dev = m_tiles_dev;
   p.k_tiles_dev = k_tiles_dev;
+  p.k_list = k_list;
+  p.k_count_dev = k_count_dev;
   p.row_map = row_map;
   p.C = C;
   p.ldc = ldc;
@@ -823,6 +844,18 @@ cudaError_t launch_tc_gemm(const void* A, int64_t lda, bool a_mn, const void* B,
   return cudaGetLastError();
 }
 
+// Column width of the sweeps' logit tiles.  256 is what the library runs: one accumulator pair
+// fills the tensor memory and the epilogue alternates with the MMAs.  The 128-column form (two
+// pairs, epilogue overlapped) is correct but measured 1.5x slower at the paper-scale shape -- its
+// MMAs are bound by operand traffic -- and is only instantiated in development builds.
+#ifdef ADWIN_DEV_EXPORTS
+#define ADWIN_SWEEP_128 1
+#else
+#define ADWIN_SWEEP_128 0
+#endif
+static int g_sweep_bn = 256;
+void set_sweep_tile_columns(int bn) { g_sweep_bn = (ADWIN_SWEEP_128 && bn == 128) ? 128 : 256; }
+
 size_t lmhead_workspace_bytes(int64_t B, int64_t T, int64_t V, int64_t ds, int64_t dt,
                               int64_t max_rows, bool want_grad, bool range_full) {
   return lm_layout(B, T, V, ds, dt, max_rows, want_grad, range_full).total;
@@ -834,8 +867,9 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
                           const int32_t* window, const int32_t* rollout_len, float alpha, int mode,
                           int flags, void* dH, int dh_dtype, float* dW, float* kl, float* logratio,
                           float* gsq, float* lse_s, float* lse_t, void* workspace,
-                          int64_t max_rows, int32_t* status, int sm_count, cudaStream_t s) {
-  const bool want_grad = dH != nullptr || dW != nullptr;
+                          int64_t max_rows, int32_t* status, int sm_count, cudaStream_t s,
+                          bool keep_G) {
+  const bool want_grad = dH != nullptr || dW != nullptr || keep_G;
   const bool range_full = (flags & ADWIN_RANGE_FULL) != 0;
   const LmLayout L = lm_layout(B, T, V, ds, dt, max_rows, want_grad, range_full);
   char* wb = static_cast<char*>(workspace);
@@ -872,9 +906,10 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
                                                 hdr, tiles, tokens, tok);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
+  const int bn = g_sweep_bn;
   CUtensorMap m_hs, m_ws, m_ht, m_wt;
-  if (!make_map(&m_hs, hs_c, ds, rows_cap, ds, kBM) || !make_map(&m_ws, ws, ds, V, ds, kBN) ||
-      !make_map(&m_ht, ht_c, dt, rows_cap, dt, kBM) || !make_map(&m_wt, wt, dt, V, dt, kBN))
+  if (!make_map(&m_hs, hs_c, ds, rows_cap, ds, kBM) || !make_map(&m_ws, ws, ds, V, ds, bn) ||
+      !make_map(&m_ht, ht_c, dt, rows_cap, dt, kBM) || !make_map(&m_wt, wt, dt, V, dt, bn))
     return cudaErrorInvalidValue;
 
   SweepParams sp;
@@ -886,7 +921,7 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
   sp.V = V;
   sp.ks_blocks = (int)((ds + kBK - 1) / kBK);
   sp.kt_blocks = (int)((dt + kBK - 1) / kBK);
-  sp.n_chunks = L.n_chunks;
+  sp.n_chunks = (int)((V + bn - 1) / bn);
   sp.n_groups = L.n_groups;
   sp.part = part;
   sp.info = info;
@@ -895,8 +930,25 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
   sp.max_tiles = L.max_tiles;
   sp.limit_ns = handshake_wait_limit_ns();
   sp.status = status;
-  if ((e = opt_in_smem(lm_sweep_kernel<false, true>)) != cudaSuccess) return e;
-  lm_sweep_kernel<false, true><<<sm_count, kThreads, kSmemBytes, s>>>(m_hs, m_ws, m_ht, m_wt, sp);
+#define ADWIN_LAUNCH_SWEEP(G_, U_, MA, MB, MC, MD)                                              \
+  do {                                                                                         \
+    if (ADWIN_SWEEP_128 && bn == 128) {                                                        \
+      if ((e = opt_in_smem(lm_sweep_kernel<G_, U_, ADWIN_SWEEP_128 ? 128 : 256>)) != cudaSuccess) return e; \
+      lm_sweep_kernel<G_, U_, ADWIN_SWEEP_128 ? 128 : 256><<<sm_count, kThreads, kSmemBytes, s>>>(MA, MB, MC, MD, sp); \
+    } else {                                                                                   \
+      if ((e = opt_in_smem(lm_sweep_kernel<G_, U_, 256>)) != cudaSuccess) return e;            \
+      lm_sweep_kernel<G_, U_, 256><<<sm_count, kThreads, kSmemBytes, s>>>(MA, MB, MC, MD, sp); \
+    }                                                                                          \
+  } while (0)
+  // the single-sweep moments are only needed for rows whose gsq does not come from sweep 2
+  const bool moments = gsq != nullptr && (!want_grad || range_full);
+  if (moments || bn != 256) {
+    ADWIN_LAUNCH_SWEEP(false, true, m_hs, m_ws, m_ht, m_wt);
+  } else {
+    if ((e = opt_in_smem(lm_sweep_kernel<false, true, 256, false>)) != cudaSuccess) return e;
+    lm_sweep_kernel<false, true, 256, false><<<sm_count, kThreads, kSmemBytes, s>>>(m_hs, m_ws, m_ht,
+                                                                                    m_wt, sp);
+  }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
   MergeParams mp;
@@ -925,16 +977,14 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
   CUtensorMap m_hg = m_hs;
   if (range_full && !make_map(&m_hg, hs_g, ds, rows_cap, ds, kBM)) return cudaErrorInvalidValue;
   if (mode == ADWIN_GRAD_FULL_KL) {
-    if ((e = opt_in_smem(lm_sweep_kernel<true, true>)) != cudaSuccess) return e;
     // With ADWIN_RANGE_FULL the compact teacher copy is in tile order and sweep 1 is done with it:
     // gather the gradient tiles' rows into the same buffer.
     if (range_full)
       lm_gather_kernel<<<gather_blocks, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(ht), T, dt,
                                                      hdr, tiles, g2t, true, ht_c);
-    lm_sweep_kernel<true, true><<<sm_count, kThreads, kSmemBytes, s>>>(m_hg, m_ws, m_ht, m_wt, sp);
+    ADWIN_LAUNCH_SWEEP(true, true, m_hg, m_ws, m_ht, m_wt);
   } else {
-    if ((e = opt_in_smem(lm_sweep_kernel<true, false>)) != cudaSuccess) return e;
-    lm_sweep_kernel<true, false><<<sm_count, kThreads, kSmemBytes, s>>>(m_hg, m_ws, m_ht, m_wt, sp);
+    ADWIN_LAUNCH_SWEEP(true, false, m_hg, m_ws, m_ht, m_wt);
   }
   if (gsq) lm_gsq_kernel<<<(unsigned)L.max_tiles, kBM, 0, s>>>(hdr, part, rowdst, L.n_groups, gsq);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
@@ -956,6 +1006,201 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
+}
+
+// ---------------------------------------------------------------------------- weight-space audit
+// Prefix-versus-full cosine of Section 4.2 in the space of the student's LM-head weight.  The
+// candidate lengths L_0 < ... < L_{K-1} (multiples of 64) cut every rollout into K+1 bins of
+// positions; dW_bin[i] = G[bin i]^T H_s[bin i] is one GEMM per bin over that bin's 64-row k-blocks,
+// the prefix gradient of candidate j is the sum of bins 0..j and the full-horizon reference the sum
+// of all bins, so the K cosines come from one pass over the K+1 bin matrices.
+constexpr int kMaxCand = 16;
+struct CandList {
+  int32_t K;
+  int32_t L[kMaxCand];
+};
+
+namespace {
+
+// k-block lists per bin: entry = first compact gradient row of a 64-row block.
+__global__ void lm_bins_kernel(const int32_t* hdr, const int32_t* __restrict__ tiles,
+                               const int32_t* __restrict__ g2t, CandList cand, int64_t list_stride,
+                               int32_t* lists, int32_t* counts) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  for (int i = 0; i <= cand.K; ++i) counts[i] = 0;
+  const int n_gt = hdr[1];
+  for (int g = 0; g < n_gt; ++g) {
+    const int32_t* e = tiles + (int64_t)g2t[g] * kTileFields;
+    for (int h = 0; h < 2; ++h) {
+      if (64 * h >= e[3]) continue;          // no gradient row in this half
+      const int t = e[1] + 64 * h;
+      int bin = 0;
+      while (bin < cand.K && cand.L[bin] <= t) ++bin;
+      lists[bin * list_stride + counts[bin]++] = g * kBM + 64 * h;
+    }
+  }
+}
+
+// Per block: sums over its share of the elements of  pre_j * full,  pre_j^2  (j < K)  and full^2,
+// where pre_j = sum of bins 0..j and full = sum of all bins.  Fixed order inside the block.
+constexpr int kGramThreads = 256;
+__global__ void __launch_bounds__(kGramThreads) lm_gram_kernel(const float* __restrict__ bins,
+                                                               int64_t n_elem, int K,
+                                                               double* partial) {
+  // fully unrolled over the compile-time bound with run-time guards, so that the accumulators
+  // stay in registers
+  double acc[2 * kMaxCand + 1];
+#pragma unroll
+  for (int i = 0; i < 2 * kMaxCand + 1; ++i) acc[i] = 0.0;
+  for (int64_t e = (int64_t)blockIdx.x * kGramThreads + threadIdx.x; e < n_elem;
+       e += (int64_t)gridDim.x * kGramThreads) {
+    float pre[kMaxCand + 1];
+    float run = 0.f;
+#pragma unroll
+    for (int i = 0; i <= kMaxCand; ++i) {
+      if (i <= K) run += bins[(int64_t)i * n_elem + e];
+      pre[i] = run;
+    }
+    const double full = (double)run;
+#pragma unroll
+    for (int j = 0; j < kMaxCand; ++j) {
+      if (j < K) {
+        acc[2 * j] += (double)pre[j] * full;
+        acc[2 * j + 1] += (double)pre[j] * (double)pre[j];
+      }
+    }
+    acc[2 * kMaxCand] += full * full;
+  }
+  __shared__ double red[kGramThreads];
+#pragma unroll
+  for (int i = 0; i < 2 * kMaxCand + 1; ++i) {
+    if (i >= 2 * K && i != 2 * kMaxCand) continue;     // unused slots (uniform across the block)
+    red[threadIdx.x] = acc[i];
+    __syncthreads();
+    for (int o = kGramThreads / 2; o > 0; o >>= 1) {
+      if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) partial[(int64_t)blockIdx.x * (2 * kMaxCand + 1) + i] = red[0];
+    __syncthreads();
+  }
+}
+
+// batch_stats[j] = { rho_w(L_j), snr, admissible (0/1), n_tokens }; L_next; flags.
+__global__ void lm_align_finish_kernel(const double* __restrict__ partial, int n_blocks,
+                                       CandList cand, double rho_star,
+                                       const int32_t* __restrict__ rollout_len, int64_t B,
+                                       int64_t T, double* batch_stats, int32_t* L_next,
+                                       int32_t* flags_out) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  const int K = cand.K;
+  double tot[2 * kMaxCand + 1];
+  for (int i = 0; i < 2 * kMaxCand + 1; ++i) {
+    double a = 0.0;
+    if (i < 2 * K || i == 2 * kMaxCand)
+      for (int b = 0; b < n_blocks; ++b) a += partial[(int64_t)b * (2 * kMaxCand + 1) + i];
+    tot[i] = a;
+  }
+  int flags = 0, best = -1;
+  const double nf = tot[2 * kMaxCand];
+  for (int j = 0; j < K; ++j) {
+    double rho;
+    if (!(nf > 0.0)) {
+      rho = 1.0;
+      flags |= ADWIN_ALIGN_DEGENERATE;
+    } else {
+      rho = tot[2 * j + 1] > 0.0 ? tot[2 * j] / (sqrt(tot[2 * j + 1]) * sqrt(nf)) : 0.0;
+    }
+    double ntok = 0.0;
+    for (int64_t b = 0; b < B; ++b) {
+      int64_t R = rollout_len ? rollout_len[b] : T;
+      R = R < 0 ? 0 : (R > T ? T : R);
+      ntok += (double)(cand.L[j] < R ? cand.L[j] : R);
+    }
+    const double r2 = rho * rho;
+    batch_stats[j * 4 + 0] = rho;
+    batch_stats[j * 4 + 1] = r2 < 1.0 ? r2 / (1.0 - r2) : INFINITY;
+    batch_stats[j * 4 + 2] = rho >= rho_star ? 1.0 : 0.0;
+    batch_stats[j * 4 + 3] = ntok;
+    if (rho >= rho_star && best < 0) best = cand.L[j];   // candidates ascend: the first is the shortest
+  }
+  if (best < 0) {
+    best = cand.L[K - 1];
+    flags |= ADWIN_ALIGN_NONE_ADMISSIBLE;
+  }
+  *L_next = best;
+  *flags_out = flags;
+}
+
+struct AlignLayout {
+  size_t off_lists, off_counts, off_bins, off_partial, total;
+  int64_t list_stride;
+  int gram_blocks;
+};
+
+AlignLayout align_layout(const LmLayout& L, int64_t V, int64_t ds, int K) {
+  auto up = [](size_t x) { return (x + 1023) & ~size_t(1023); };
+  AlignLayout A;
+  A.list_stride = 2 * L.max_tiles;
+  A.gram_blocks = 1184;
+  size_t o = L.total;
+  A.off_lists = o;    o = up(o + (size_t)(K + 1) * A.list_stride * 4);
+  A.off_counts = o;   o = up(o + (size_t)(K + 1) * 4);
+  A.off_bins = o;     o = up(o + (size_t)(K + 1) * (size_t)V * ds * 4);
+  A.off_partial = o;  o = up(o + (size_t)A.gram_blocks * (2 * kMaxCand + 1) * 8);
+  A.total = o;
+  return A;
+}
+
+}  // namespace
+
+size_t lmhead_align_workspace_bytes(int64_t B, int64_t T, int64_t V, int64_t ds, int64_t dt,
+                                    int64_t max_rows, int K) {
+  return align_layout(lm_layout(B, T, V, ds, dt, max_rows, true, false), V, ds, K).total;
+}
+
+cudaError_t launch_lmhead_weight_align(const void* hs, const void* ws, const void* ht,
+                                       const void* wt, int64_t B, int64_t T, int64_t V, int64_t ds,
+                                       int64_t dt, const int32_t* tokens,
+                                       const int32_t* rollout_len, const int32_t* cand_host, int K,
+                                       double rho_star, int mode, float* kl, float* logratio,
+                                       float* gsq, double* batch_stats, int32_t* L_next,
+                                       int32_t* flags_out, void* workspace, int64_t max_rows,
+                                       int32_t* status, int sm_count, cudaStream_t s) {
+  const LmLayout L = lm_layout(B, T, V, ds, dt, max_rows, true, false);
+  const AlignLayout A = align_layout(L, V, ds, K);
+  char* wb = static_cast<char*>(workspace);
+  // every position of every rollout carries gradient here: the window is the rollout itself
+  // (window == NULL stands for W_b = T in the row map, so E_b = R_b)
+  cudaError_t e = launch_lmhead(hs, ws, ht, wt, B, T, V, ds, dt, tokens, nullptr, rollout_len, 1.0f,
+                                mode, 0, nullptr, ADWIN_F32, nullptr, kl, logratio, gsq, nullptr,
+                                nullptr, workspace, max_rows, status, sm_count, s, true);
+  if (e != cudaSuccess) return e;
+  const int32_t* hdr = reinterpret_cast<const int32_t*>(wb + L.off_hdr);
+  const int32_t* tiles = reinterpret_cast<const int32_t*>(wb + L.off_tiles);
+  const int32_t* g2t = reinterpret_cast<const int32_t*>(wb + L.off_g2t);
+  const __nv_bfloat16* hs_c = reinterpret_cast<const __nv_bfloat16*>(wb + L.off_hs);
+  const __nv_bfloat16* G = reinterpret_cast<const __nv_bfloat16*>(wb + L.off_G);
+  int32_t* lists = reinterpret_cast<int32_t*>(wb + A.off_lists);
+  int32_t* counts = reinterpret_cast<int32_t*>(wb + A.off_counts);
+  float* bins = reinterpret_cast<float*>(wb + A.off_bins);
+  double* partial = reinterpret_cast<double*>(wb + A.off_partial);
+  CandList cand;
+  cand.K = K;
+  for (int i = 0; i < kMaxCand; ++i) cand.L[i] = i < K ? cand_host[i] : 0;
+  lm_bins_kernel<<<1, 32, 0, s>>>(hdr, tiles, g2t, cand, A.list_stride, lists, counts);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  const int64_t rows_cap = L.max_tiles * kBM;
+  for (int i = 0; i <= K; ++i) {
+    e = launch_tc_gemm(G, L.ldG, true, hs_c, ds, true, V, ds, rows_cap,
+                       bins + (size_t)i * V * ds, ds, false, nullptr, nullptr, nullptr, status,
+                       sm_count, s, lists + (size_t)i * A.list_stride, counts + i);
+    if (e != cudaSuccess) return e;
+  }
+  lm_gram_kernel<<<A.gram_blocks, kGramThreads, 0, s>>>(bins, V * ds, K, partial);
+  lm_align_finish_kernel<<<1, 32, 0, s>>>(partial, A.gram_blocks, cand, rho_star, rollout_len, B, T,
+                                          batch_stats, L_next, flags_out);
+  return cudaGetLastError();
 }
 
 }  // namespace adwin

@@ -48,7 +48,7 @@ __global__ void __launch_bounds__(kMapThreads) rowmap_kernel(
     for (int64_t b = b0; b < b1; ++b) {
       int E, P;
       bool bad;
-      clamp_lengths(window[b], rollout_len ? rollout_len[b] : (int32_t)T, T, flags, E, P, bad);
+      clamp_lengths(window ? window[b] : (int32_t)T, rollout_len ? rollout_len[b] : (int32_t)T, T, flags, E, P, bad);
       any_bad |= bad;
       range[b] = P;
       ewin[b] = E;
@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(kMapThreads) rowmap_kernel(
     const int t = (int)(i - b * T);
     int E, P;
     bool bad;
-    clamp_lengths(window[b], rollout_len ? rollout_len[b] : (int32_t)T, T, flags, E, P, bad);
+    clamp_lengths(window ? window[b] : (int32_t)T, rollout_len ? rollout_len[b] : (int32_t)T, T, flags, E, P, bad);
     if (t >= P && ADWIN_CHK(b < B && t >= 0 && t < T, status)) {
       kl[i] = 0.f;
       logratio[i] = 0.f;

@@ -28,6 +28,7 @@ constexpr int kBN = 256;            // columns of an MMA tile (TMEM columns of o
 constexpr int kBK = 64;             // bf16 per k-block (one 128-byte swizzle span)
 constexpr int kUmmaK = 16;          // K of one tcgen05.mma (bf16)
 constexpr int kStages = 4;
+constexpr int kMaxStages = 6;        // barrier arrays are sized for the deepest pipeline in use
 constexpr int kABytes = kBM * kBK * 2;            // 16384
 constexpr int kBBytes = kBN * kBK * 2;            // 32768
 constexpr int kStageBytes = kABytes + kBBytes;    // 49152
@@ -42,8 +43,8 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
 // Control block at the start of dynamic shared memory; the stages follow at the next 1024-byte
 // boundary.
 struct Ctrl {
-  unsigned long long full[kStages];    // TMA -> MMA: the stage's tiles have landed
-  unsigned long long empty[kStages];   // MMA -> TMA: the stage's tiles have been consumed
+  unsigned long long full[kMaxStages];   // TMA -> MMA: the stage's tiles have landed
+  unsigned long long empty[kMaxStages];  // MMA -> TMA: the stage's tiles have been consumed
   unsigned long long acc_full[2];      // MMA -> epilogue: accumulator slot complete
   unsigned long long acc_empty[2];     // epilogue -> MMA: accumulator slot read out
   unsigned long long drain;            // give-up path: all issued MMAs have retired
@@ -209,9 +210,9 @@ constexpr uint32_t kStepMNMajor = (kUmmaK * 128) >> 4;     // 16 k-rows of 128 b
 // Instruction descriptor of tcgen05.mma.kind::f16 for bf16 x bf16 -> fp32, M = 128, N = 256:
 // accumulator format fp32 (bits 4..5 = 1), A and B format bf16 (bits 7..9, 10..12 = 1), operand
 // majors in bits 15 / 16 (0 = K-major, 1 = MN-major), N >> 3 in bits 17..22, M >> 4 in bits 24..28.
-__host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn) {
+__host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn, int n = kBN) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-         ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 }
 __device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc,
                                      uint32_t idesc, uint32_t accumulate) {
@@ -230,10 +231,10 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 }
 
 // The four MMAs of one k-block.  `first` clears the accumulator on the very first MMA of a tile.
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, int N = kBN>
 __device__ __forceinline__ void issue_kblock(uint32_t tmem_d, uint32_t a_saddr, uint32_t b_saddr,
                                              bool first) {
-  constexpr uint32_t idesc = instr_desc(A_MN, B_MN);
+  constexpr uint32_t idesc = instr_desc(A_MN, B_MN, N);
   const uint64_t ad = A_MN ? desc_mn_major(a_saddr) : desc_k_major(a_saddr);
   const uint64_t bd = B_MN ? desc_mn_major(b_saddr) : desc_k_major(b_saddr);
 #pragma unroll
