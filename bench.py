@@ -47,6 +47,8 @@ def parse():
     ap.add_argument("--seqs", type=int, default=None, help="override B (profiling a small case only)")
     ap.add_argument("--positions", type=int, default=None,
                     help="override T (profiling a small case only)")
+    ap.add_argument("--sustained-seconds", type=float, default=2.2,
+                    help="length of the back-to-back run with sampled clocks (0 = skip)")
     ap.add_argument("--no-side", action="store_true",
                     help="skip the side measurements (profiling a small case only)")
     ap.add_argument("--lmhead-seqs", type=int, default=None,
@@ -72,7 +74,7 @@ def measured_peak():
 # ends, a residue bounded by the L2 size that does not grow with the rows, so at full size the
 # writes are taken as the gradient bytes themselves.
 TRAFFIC_READ_BYTES_PER_ROW = 611598
-TRAFFIC_KERNEL_SHA = "63b30a9d15568918"
+TRAFFIC_KERNEL_SHA = "18f9a1f9922e75ed"
 
 
 def recorded_traffic(rows, V):
@@ -346,8 +348,8 @@ def run_ours(args):
     # ---- the same step back to back for >= 2 s with the clocks sampled: what the kernel does once
     # the SM clock has settled under sustained load (nothing is set, only read)
     sustained = None
-    if side:
-        n_sus = max(50, int(2200.0 / max(ms_step, 1e-3)))
+    if side and args.sustained_seconds > 0:
+        n_sus = max(50, int(1e3 * args.sustained_seconds / max(ms_step, 1e-3)))
         sus_sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
         sus_sampler.start()
         time.sleep(0.2)
