@@ -440,6 +440,7 @@ int adwin_lmhead_weight_align(const void* hidden_student, const void* w_student,
 
 #ifdef ADWIN_DEV_EXPORTS
 void adwin_dev_set_sweep_bn(int bn) { set_sweep_tile_columns(bn); }
+void adwin_dev_set_sweep_pair(int on) { set_sweep_pair(on); }
 // Development build only: the tensor-core GEMM on its own, C = A B (bf16 in, fp32 or bf16 out).
 int adwin_dev_gemm(const void* A, int64_t lda, int a_mn, const void* Bm, int64_t ldb, int b_mn,
                    int64_t M, int64_t N, int64_t K, void* C, int64_t ldc, int c_bf16,

@@ -66,6 +66,7 @@ cudaError_t launch_drift_curves(const float* entropy, const int32_t* rank,
 
 // Fused LM-head form (lmhead.cu).
 void set_sweep_tile_columns(int bn);
+void set_sweep_pair(int on);
 size_t lmhead_workspace_bytes(int64_t B, int64_t T, int64_t V, int64_t ds, int64_t dt,
                               int64_t max_rows, bool want_grad, bool range_full);
 cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const void* wt, int64_t B,

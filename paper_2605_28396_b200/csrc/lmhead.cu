@@ -277,7 +277,7 @@ __device__ __forceinline__ void group_chunks(const SweepParams& p, int g, int& c
 // gsq from sweep 2, or no gsq is asked for).
 // GRAD = false: sweep 1 (statistics).  GRAD = true: sweep 2 (logit gradient); NEED_U = false
 // skips the teacher product there (the sampled-token estimator of Eq. 4 does not need it).
-template <bool GRAD, bool NEED_U, int BN, bool MOMENTS = true>
+template <bool GRAD, bool NEED_U, int BN, bool MOMENTS = true, bool PAIR = false>
 __global__ void __launch_bounds__(kThreads, 1)
 lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constant__ CUtensorMap map_ws,
                 const __grid_constant__ CUtensorMap map_ht, const __grid_constant__ CUtensorMap map_wt,
@@ -285,8 +285,14 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
   // BN = 256: one accumulator pair (student + teacher tile) fills the 512 TMEM columns, the
   // epilogue and the MMAs of the next chunk alternate.  BN = 128: two pairs, so the epilogue of a
   // chunk overlaps the MMAs of the next, at 1.5x the operand bytes per flop.
-  constexpr int kSt = BN == 256 ? 4 : 6;            // pipeline stages
-  constexpr int kStB = kABytes + BN * kBK * 2;      // bytes per stage
+  // PAIR: two CTAs of a cluster form one MMA unit (cta_group::2): a 256-row tile pair, each CTA
+  // stages its own A tile and half of the B tile (32 KB per stage instead of 48) and reads its own
+  // 128 rows of the accumulators; the even CTA issues the MMAs.
+  static_assert(!PAIR || BN == 256, "the pair form uses 256-column tiles");
+  constexpr int kBrows = PAIR ? BN / 2 : BN;        // rows of the B tile this CTA stages
+  constexpr int kStB = kABytes + kBrows * kBK * 2;  // bytes per stage
+  constexpr int kSt = (kStages * kStageBytes) / kStB < kMaxStages ? (kStages * kStageBytes) / kStB
+                                                                  : kMaxStages;   // pipeline stages
   constexpr int kAcc = kTmemCols / (2 * BN);        // accumulator pairs
   constexpr int kHalf = BN / 2;                     // columns per epilogue warpgroup
   static_assert(kSt <= kMaxStages && kSt * kStB <= kStages * kStageBytes, "stage budget");
@@ -295,6 +301,7 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
   const uint32_t stage0 = (smem_addr(smem_raw) + kCtrlBytes + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort = &ctrl->abort;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // 0: the CTA that issues the MMAs
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSt; ++s) {
@@ -303,31 +310,43 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
     }
     for (int s = 0; s < kAcc; ++s) {
       bar_init(smem_addr(&ctrl->acc_full[s]), 1);
-      bar_init(smem_addr(&ctrl->acc_empty[s]), kEpiThreads);
+      bar_init(smem_addr(&ctrl->acc_empty[s]), PAIR ? 2 * (kEpiThreads / 32) : kEpiThreads);
     }
     bar_init(smem_addr(&ctrl->drain), 1);
     ctrl->abort = 0;
     bar_init_fence();
   }
   if (warp == 2) {
-    tmem_alloc(smem_addr(&ctrl->tmem_base), kTmemCols);
-    tmem_relinquish();
+    if (PAIR) {
+      tmem_alloc_pair(smem_addr(&ctrl->tmem_base), kTmemCols);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(smem_addr(&ctrl->tmem_base), kTmemCols);
+      tmem_relinquish();
+    }
     tc_fence_before_sync();
   }
   __syncthreads();
+  if (PAIR) cluster_sync();   // the partner's barriers exist before anything signals them
   tc_fence_after_sync();
   const uint32_t tmem_base = ctrl->tmem_base;
 
+  // Work items: (tile, vocabulary group), or (pair of consecutive tiles, group) for a CTA pair,
+  // in which CTA `rank` owns tile 2*pair + rank (the second tile of the last pair may not exist).
   const int n_tiles = p.hdr[GRAD ? 1 : 0];
-  const int64_t n_items = (int64_t)n_tiles * p.n_groups;
+  const int64_t n_units = PAIR ? (n_tiles + 1) / 2 : n_tiles;
+  const int64_t n_items = n_units * p.n_groups;
+  const int64_t first_item = PAIR ? blockIdx.x / 2 : blockIdx.x;
+  const int64_t item_step = PAIR ? gridDim.x / 2 : gridDim.x;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int64_t item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
-        const int tile = (int)(item / p.n_groups), g = (int)(item % p.n_groups);
+      for (int64_t item = first_item; ok && item < n_items; item += item_step) {
+        const int tile = (PAIR ? 2 : 1) * (int)(item / p.n_groups) + (int)rank;
+        const int g = (int)(item % p.n_groups);
         const int row0 = tile * kBM;          // compact row of the tile (tile or gradient-tile order)
         int c0, c1;
         group_chunks(p, g, c0, c1);
@@ -341,14 +360,25 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
               if (!bar_wait(smem_addr(&ctrl->empty[s]), ph ^ 1, abort, p.limit_ns)) { ok = false; break; }
               const uint32_t bar = smem_addr(&ctrl->full[s]);
               const uint32_t a = stage0 + s * kStB, b = a + kABytes;
-              bar_expect_tx(bar, kStB);
-              tma_load_2d(a, ma, kb * kBK, row0, bar);
-              tma_load_2d(b, mb, kb * kBK, c * BN, bar);
+              if (PAIR) {
+                // both CTAs' bytes are counted by the even CTA's barrier
+                if (rank == 0) bar_expect_tx(bar, 2 * kStB);
+                const uint32_t bar0 = map_to_cta(bar, 0);
+                tma_load_2d_pair(a, ma, kb * kBK, row0, bar0);
+                tma_load_2d_pair(b, mb, kb * kBK, c * BN + (int)rank * kBrows, bar0);
+              } else {
+                bar_expect_tx(bar, kStB);
+                tma_load_2d(a, ma, kb * kBK, row0, bar);
+                tma_load_2d(b, mb, kb * kBK, c * BN, bar);
+              }
             }
           }
         }
       }
-      if (!ok) {   // give up: let the copies in flight land before the CTA's shared memory goes
+      // give up: let the copies in flight land before the CTA's shared memory goes (in a pair the
+      // even CTA's barriers count both CTAs' copies, and the final cluster barrier holds the odd
+      // CTA until the even one has waited for them)
+      if (!ok && rank == 0) {
         const uint32_t n_out = it < (uint32_t)kSt ? it : (uint32_t)kSt;
         for (uint32_t j = it - n_out; j < it; ++j)
           bar_wait_drain(smem_addr(&ctrl->full[j % kSt]), (j / kSt) & 1);
@@ -356,10 +386,10 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       uint32_t it = 0, acc_it = 0;
       bool ok = true;
-      for (int64_t item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+      for (int64_t item = first_item; ok && item < n_items; item += item_step) {
         int c0, c1;
         group_chunks(p, (int)(item % p.n_groups), c0, c1);
         for (int c = c0; ok && c < c1; ++c, ++acc_it) {
@@ -374,15 +404,24 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
               if (!bar_wait(smem_addr(&ctrl->full[s]), ph, abort, p.limit_ns)) { ok = false; break; }
               tc_fence_after_sync();
               const uint32_t a = stage0 + s * kStB, b = a + kABytes;
-              issue_kblock<false, false, BN>(tmem_d, a, b, kb == 0);
-              umma_commit(smem_addr(&ctrl->empty[s]));
+              if (PAIR) {
+                issue_kblock_pair<BN>(tmem_d, a, b, kb == 0);
+                umma_commit_pair(smem_addr(&ctrl->empty[s]));
+              } else {
+                issue_kblock<false, false, BN>(tmem_d, a, b, kb == 0);
+                umma_commit(smem_addr(&ctrl->empty[s]));
+              }
             }
           }
-          if (ok) umma_commit(smem_addr(&ctrl->acc_full[slot]));
+          if (ok) {
+            if (PAIR) umma_commit_pair(smem_addr(&ctrl->acc_full[slot]));
+            else umma_commit(smem_addr(&ctrl->acc_full[slot]));
+          }
         }
       }
       if (!ok) {   // give up: wait until the MMAs already issued have retired
-        umma_commit(smem_addr(&ctrl->drain));
+        if (PAIR) umma_commit_pair(smem_addr(&ctrl->drain));
+        else umma_commit(smem_addr(&ctrl->drain));
         bar_wait_drain(smem_addr(&ctrl->drain), 0);
       }
     }
@@ -395,9 +434,11 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
     const uint32_t t_quad = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * kHalf);
     uint32_t acc_it = 0;
     bool ok = true;
-    for (int64_t item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
-      const int tile_c = (int)(item / p.n_groups), g = (int)(item % p.n_groups);
-      const int tile = GRAD ? p.g2t[tile_c] : tile_c;
+    for (int64_t item = first_item; ok && item < n_items; item += item_step) {
+      const int tile_c = (PAIR ? 2 : 1) * (int)(item / p.n_groups) + (int)rank;
+      const int g = (int)(item % p.n_groups);
+      const bool live = tile_c < n_tiles;     // the last pair's second tile may not exist
+      const int tile = !live ? 0 : (GRAD ? p.g2t[tile_c] : tile_c);
       int c0, c1;
       group_chunks(p, g, c0, c1);
 
@@ -405,8 +446,10 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
       RowAcc acc;
       float dref = 0.f, q = 0.f;   // q: this thread's share of the row's sum g^2 (sweep 2)
       float L2s = 0.f, a1 = 0.f, a0 = 0.f, gy = 0.f;
-      if (!GRAD) {
-        acc.reset();
+      acc.reset();
+      if (!live) {
+        // nothing to read: the tile's accumulators hold products of whatever the loads returned
+      } else if (!GRAD) {
         const float* tk = p.tok + ((int64_t)tile * kBM + row) * kTokFields;
         dref = tk[0] - tk[1];      // centre of z - u for this row: the sampled token's difference
       } else {
@@ -428,7 +471,7 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
         const int64_t col_base = (int64_t)c * BN + half * kHalf;
         const bool ragged = col_base + kHalf > p.V;
 #pragma unroll 1
-        for (int j = 0; j < kHalf / 32; ++j) {
+        for (int j = 0; live && j < kHalf / 32; ++j) {
           uint32_t zr[32], ur[32];
           tmem_ld32(t_lane + j * 32, zr);
           if (NEED_U) tmem_ld32(t_lane + BN + j * 32, ur);
@@ -488,11 +531,19 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
           }
         }
         tc_fence_before_sync();
-        bar_arrive(smem_addr(&ctrl->acc_empty[slot]));
+        if (PAIR) {   // one arrival per warp: the odd CTA's arrivals cross to the even CTA
+          __syncwarp();
+          if (lane == 0) {
+            if (rank != 0) bar_arrive_cluster(map_to_cta(smem_addr(&ctrl->acc_empty[slot]), 0));
+            else bar_arrive(smem_addr(&ctrl->acc_empty[slot]));
+          }
+        } else {
+          bar_arrive(smem_addr(&ctrl->acc_empty[slot]));
+        }
       }
-      if (GRAD && ok && ADWIN_CHK(tile_c < p.max_tiles && g < p.n_groups, p.status))
+      if (GRAD && ok && live && ADWIN_CHK(tile_c < p.max_tiles && g < p.n_groups, p.status))
         p.part[(((int64_t)tile_c * p.n_groups + g) * 2 + half) * kBM + row] = q;
-      if (!GRAD && ok && ADWIN_CHK(tile < p.max_tiles && g < p.n_groups && row < kBM, p.status)) {
+      if (!GRAD && ok && live && ADWIN_CHK(tile < p.max_tiles && g < p.n_groups && row < kBM, p.status)) {
         float* o = p.part + ((((int64_t)tile * p.n_groups + g) * 2 + half) * kRecFields) * kBM + row;
         o[0 * kBM] = acc.m2s;
         o[1 * kBM] = acc.S;
@@ -505,12 +556,17 @@ lm_sweep_kernel(const __grid_constant__ CUtensorMap map_hs, const __grid_constan
       }
     }
   }
-  if (*abort && threadIdx.x == 0) atomicOr(p.status, ADWIN_DEV_TIMEOUT);
+  if (*abort && threadIdx.x == 0) {
+    atomicOr(p.status, ADWIN_DEV_TIMEOUT);
+    if (PAIR) store_cluster_u32(map_to_cta(smem_addr(&ctrl->abort), rank ^ 1u), 1u);   // partner too
+  }
   tc_fence_before_sync();
   __syncthreads();
+  if (PAIR) cluster_sync();   // neither CTA leaves while the other may still use its memory
   if (warp == 2) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, kTmemCols);
+    if (PAIR) tmem_dealloc_pair(tmem_base, kTmemCols);
+    else tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
@@ -795,6 +851,29 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   }
 }
 
+// One sweep launch: single CTAs, or clusters of two for the pair form.
+template <bool GRAD, bool NEED_U, int BN, bool MOM, bool PAIR>
+cudaError_t launch_sweep(const CUtensorMap& m_hs, const CUtensorMap& m_ws, const CUtensorMap& m_ht,
+                         const CUtensorMap& m_wt, const SweepParams& sp, int sm_count,
+                         cudaStream_t s) {
+  auto kernel = lm_sweep_kernel<GRAD, NEED_U, BN, MOM, PAIR>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(PAIR ? (sm_count & ~1) : sm_count);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, m_hs, m_ws, m_ht, m_wt, sp);
+}
+
 template <typename K>
 cudaError_t opt_in_smem(K kernel) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
@@ -853,6 +932,13 @@ cudaError_t launch_tc_gemm(const void* A, int64_t lda, bool a_mn, const void* B,
 #else
 #define ADWIN_SWEEP_128 0
 #endif
+// CTA pairs (tcgen05 cta_group::2: a 256-row tile pair per MMA, each CTA staging half of the B
+// tile).  Correct (the whole test-suite passes with it) and it cuts the operand bytes a CTA pulls
+// through L2 by a third, but at the paper-scale shape it measured no faster than single CTAs
+// (44.4 ms against 42.2 ms for the statistics sweep): the partner CTAs' epilogues have to meet
+// before the next chunk's MMAs start.  Instantiated in development builds only.
+static int g_sweep_pair = 0;
+void set_sweep_pair(int on) { g_sweep_pair = (ADWIN_SWEEP_128 && on) ? 1 : 0; }
 static int g_sweep_bn = 256;
 void set_sweep_tile_columns(int bn) { g_sweep_bn = (ADWIN_SWEEP_128 && bn == 128) ? 128 : 256; }
 
@@ -930,25 +1016,27 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
   sp.max_tiles = L.max_tiles;
   sp.limit_ns = handshake_wait_limit_ns();
   sp.status = status;
-#define ADWIN_LAUNCH_SWEEP(G_, U_, MA, MB, MC, MD)                                              \
-  do {                                                                                         \
-    if (ADWIN_SWEEP_128 && bn == 128) {                                                        \
-      if ((e = opt_in_smem(lm_sweep_kernel<G_, U_, ADWIN_SWEEP_128 ? 128 : 256>)) != cudaSuccess) return e; \
-      lm_sweep_kernel<G_, U_, ADWIN_SWEEP_128 ? 128 : 256><<<sm_count, kThreads, kSmemBytes, s>>>(MA, MB, MC, MD, sp); \
-    } else {                                                                                   \
-      if ((e = opt_in_smem(lm_sweep_kernel<G_, U_, 256>)) != cudaSuccess) return e;            \
-      lm_sweep_kernel<G_, U_, 256><<<sm_count, kThreads, kSmemBytes, s>>>(MA, MB, MC, MD, sp); \
-    }                                                                                          \
-  } while (0)
+  // 128-row boxes of the output embeddings for the pair form (each CTA stages half a B tile)
+  const bool pair = ADWIN_SWEEP_128 && g_sweep_pair && bn == 256 && sm_count >= 2;
+  CUtensorMap m_ws_h = m_ws, m_wt_h = m_wt;
+  if (pair && (!make_map(&m_ws_h, ws, ds, V, ds, kBN / 2) || !make_map(&m_wt_h, wt, dt, V, dt, kBN / 2)))
+    return cudaErrorInvalidValue;
   // the single-sweep moments are only needed for rows whose gsq does not come from sweep 2
   const bool moments = gsq != nullptr && (!want_grad || range_full);
-  if (moments || bn != 256) {
-    ADWIN_LAUNCH_SWEEP(false, true, m_hs, m_ws, m_ht, m_wt);
+  if (bn != 256) {
+#if ADWIN_SWEEP_128
+    e = launch_sweep<false, true, 128, true, false>(m_hs, m_ws, m_ht, m_wt, sp, sm_count, s);
+#endif
+#if ADWIN_SWEEP_128
+  } else if (pair) {
+    e = moments ? launch_sweep<false, true, 256, true, true>(m_hs, m_ws_h, m_ht, m_wt_h, sp, sm_count, s)
+                : launch_sweep<false, true, 256, false, true>(m_hs, m_ws_h, m_ht, m_wt_h, sp, sm_count, s);
+#endif
   } else {
-    if ((e = opt_in_smem(lm_sweep_kernel<false, true, 256, false>)) != cudaSuccess) return e;
-    lm_sweep_kernel<false, true, 256, false><<<sm_count, kThreads, kSmemBytes, s>>>(m_hs, m_ws, m_ht,
-                                                                                    m_wt, sp);
+    e = moments ? launch_sweep<false, true, 256, true, false>(m_hs, m_ws, m_ht, m_wt, sp, sm_count, s)
+                : launch_sweep<false, true, 256, false, false>(m_hs, m_ws, m_ht, m_wt, sp, sm_count, s);
   }
+  if (e != cudaSuccess) return e;
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
   MergeParams mp;
@@ -982,10 +1070,31 @@ cudaError_t launch_lmhead(const void* hs, const void* ws, const void* ht, const 
     if (range_full)
       lm_gather_kernel<<<gather_blocks, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(ht), T, dt,
                                                      hdr, tiles, g2t, true, ht_c);
-    ADWIN_LAUNCH_SWEEP(true, true, m_hg, m_ws, m_ht, m_wt);
+    if (bn != 256) {
+#if ADWIN_SWEEP_128
+      e = launch_sweep<true, true, 128, true, false>(m_hg, m_ws, m_ht, m_wt, sp, sm_count, s);
+#endif
+#if ADWIN_SWEEP_128
+    } else if (pair) {
+      e = launch_sweep<true, true, 256, true, true>(m_hg, m_ws_h, m_ht, m_wt_h, sp, sm_count, s);
+#endif
+    } else {
+      e = launch_sweep<true, true, 256, true, false>(m_hg, m_ws, m_ht, m_wt, sp, sm_count, s);
+    }
   } else {
-    ADWIN_LAUNCH_SWEEP(true, false, m_hg, m_ws, m_ht, m_wt);
+    if (bn != 256) {
+#if ADWIN_SWEEP_128
+      e = launch_sweep<true, false, 128, true, false>(m_hg, m_ws, m_ht, m_wt, sp, sm_count, s);
+#endif
+#if ADWIN_SWEEP_128
+    } else if (pair) {
+      e = launch_sweep<true, false, 256, true, true>(m_hg, m_ws_h, m_ht, m_wt_h, sp, sm_count, s);
+#endif
+    } else {
+      e = launch_sweep<true, false, 256, true, false>(m_hg, m_ws, m_ht, m_wt, sp, sm_count, s);
+    }
   }
+  if (e != cudaSuccess) return e;
   if (gsq) lm_gsq_kernel<<<(unsigned)L.max_tiles, kBM, 0, s>>>(hdr, part, rowdst, L.n_groups, gsq);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
 

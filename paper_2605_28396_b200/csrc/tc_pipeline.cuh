@@ -258,5 +258,86 @@ __device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap* ma
   }
 }
 
+// ---------------------------------------------------------------------------- CTA pairs
+// Forms used when two CTAs of a cluster work as one MMA unit (cta_group::2): an MMA tile is then
+// 256 rows (128 per CTA, each CTA's rows accumulate in its own tensor memory) x 256 columns, and
+// each CTA stages only half of the B tile, so the operand bytes per flop that a CTA pulls through
+// L2 drop by a third.  The even CTA of the pair (cluster rank 0) issues the MMAs; TMA loads of both
+// CTAs report their bytes to its `full` barrier; tcgen05.commit signals barriers at the same
+// shared-memory offset in both CTAs.  No load is multicast: each CTA fetches its own tiles.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::
+                   : "memory");
+}
+__device__ __forceinline__ void bar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr)
+               : "memory");
+}
+__device__ __forceinline__ void store_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),
+               "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols)
+               : "memory");
+}
+// TMA load of a CTA of a pair; `bar_cluster` is the shared::cluster address of the barrier that
+// receives the bytes (the even CTA's).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int32_t c0,
+                                                 int32_t c1, uint32_t bar_cluster) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+      "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void umma_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrive on the barrier at this shared-memory offset in both CTAs of the pair once every
+// tcgen05.mma issued so far has retired.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 "
+      "[%0], %1;" ::"r"(bar),
+      "h"(mask)
+      : "memory");
+}
+// The four MMAs of one k-block of a pair tile (K-major operands, M = 256).
+template <int N>
+__device__ __forceinline__ void issue_kblock_pair(uint32_t tmem_d, uint32_t a_saddr,
+                                                  uint32_t b_saddr, bool first) {
+  constexpr uint32_t idesc = (instr_desc(false, false, N) & ~(0x1fu << 24)) | ((256u >> 4) << 24);
+  const uint64_t ad = desc_k_major(a_saddr), bd = desc_k_major(b_saddr);
+#pragma unroll
+  for (int k = 0; k < kBK / kUmmaK; ++k)
+    umma_pair(tmem_d, ad + (uint64_t)(k * kStepKMajor), bd + (uint64_t)(k * kStepKMajor), idesc,
+              (first && k == 0) ? 0u : 1u);
+}
+
 }  // namespace tc
 }  // namespace adwin
