@@ -559,7 +559,31 @@ def run_ours(args):
                    "launches_per_step": 9,
                    "path": "adwin_opd_kl_lmhead_fwd_bwd: rowmap, plan, 2 gathers, lm_sweep "
                            "(statistics), merge, lm_sweep (gradient), tc_gemm (dH_s), tc_gemm (dW_s)"}
-        del lb, dH, dW, lws
+        # the audit in the space of the LM-head weight on the same batch (every position of every
+        # rollout carries gradient; the paper's candidate list)
+        del dH, dW, lws
+        torch.cuda.empty_cache()
+        allrows = int(lb.rollout_len.sum())
+        aws = torch.empty(int(api.lib().adwin_lmhead_align_workspace_bytes(LB, LT, V, ds, dt, allrows, 6))
+                          + 1024, dtype=torch.uint8, device=dev)
+        al_out = None
+
+        def align_step():
+            nonlocal al_out
+            al_out = api.adwin_lmhead_weight_align(lb.hidden_student, lb.w_student,
+                                                   lb.hidden_teacher, lb.w_teacher, lb.tokens,
+                                                   lb.rollout_len, None, 0.0, max_rows=allrows,
+                                                   workspace=aws, dev_status=status)
+        al_ms = time_loop(align_step, 2, warm=1)
+        fl_al = 2.0 * (2.0 * allrows * V * (ds + dt)) + 2.0 * allrows * V * ds
+        lm_line["weight_align"] = {
+            "positions": allrows, "candidates": list(api.DEFAULT_CANDIDATES), "ms_per_step": al_ms,
+            "method_flops": fl_al, "achieved_tflops": fl_al / (al_ms * 1e-3) / 1e12,
+            "rho_w": [float(x) for x in al_out.batch_stats[:, 0].cpu()],
+            "L_next": int(al_out.L_next.item()), "steps": 2,
+            "path": "adwin_lmhead_weight_align: fused pass over every position (2 sweeps), 7 bin "
+                    "GEMMs, one pass over the bin matrices"}
+        del lb, aws
         torch.cuda.empty_cache()
 
     # ---- end to end through the host-buffer entry point (copies inside the timed region)
