@@ -73,6 +73,7 @@ struct StagedPlan {
   int num_clusters;
   uint32_t slot_bytes;    // 2 * chunk_pieces * 16
   uint64_t wait_limit_ns; // limit of the handshake waits (the drain loops keep kWaitLimitNs)
+  int tm;                 // 1: streamed chunks are kept in tensor memory between the sweeps
 };
 
 // What the consumers need to know about a row: which global row it is, whether its gradient is
@@ -100,6 +101,8 @@ struct __align__(16) Ctrl {
   float xbuf[2][kMaxRec][8];   // per row parity: one record per (rank, warp)
   float sbuf[kMaxRec][8];      // records of the running-maximum fallback
   int16_t tab[kMaxChunks];     // chunk j -> resident slot k (>= 0) or -1 (streamed)
+  int16_t ord[kMaxChunks];     // chunk j -> its ordinal among the streamed chunks
+  uint32_t tmem_base;          // tensor-memory allocation (TM mode)
   RowMeta meta[kMetaDepth];    // row metadata, filled a few rows ahead by the metadata lane
   unsigned long long meta_full[kMetaDepth];
   unsigned long long meta_empty[kMetaDepth];
@@ -213,6 +216,32 @@ __device__ __forceinline__ uint64_t global_timer() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
+
+// Tensor memory as a scratchpad (TM mode): 512 columns x 128 lanes x 32 bit = 256 KB per SM that a
+// kernel without MMAs leaves idle.  A consumer thread parks the 16-byte pieces it has read in
+// sweep 1 in its own lane (lane = 32*(warp%4) + laneid, the only lanes a warp may touch) and gets
+// them back in sweep 2, so the streamed chunks are neither kept in shared memory nor fetched again.
+constexpr int kTmCols = 512;
+constexpr int kTmColsPerThread = 128;      // four consumer warps share the 512 columns of a lane group
+__device__ __forceinline__ void tm_alloc(uint32_t dst_smem) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(kTmCols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tm_dealloc(uint32_t taddr) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(kTmCols) : "memory");
+}
+__device__ __forceinline__ void tm_store8(uint32_t taddr, const uint4& a, const uint4& b) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr),
+               "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
+}
+__device__ __forceinline__ void tm_load8(uint32_t taddr, uint4& a, uint4& b) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w)
+               : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tm_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tm_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Bounded wait of one thread.  Returns immediately (false) once the CTA has given up.
 template <bool CLUSTER>
@@ -475,7 +504,7 @@ __device__ __forceinline__ float lane_sum(float v) {
   return v;
 }
 
-template <typename TIn, typename TOut>
+template <typename TIn, typename TOut, bool TM>
 __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, StagedPlan plan) {
   constexpr int N = Elem<TIn>::N;
   constexpr int NP = Pairs<TIn>::NP;
@@ -512,7 +541,11 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
       mbar_init(smem_u32(&ctrl.ring_full[s]), 1);
       mbar_init(smem_u32(&ctrl.ring_empty[s]), kNW);
     }
-    for (int j = 0; j < nch; ++j) ctrl.tab[j] = (int16_t)resident_slot(j, nres, nch);
+    for (int j = 0, o = 0; j < nch; ++j) {
+      ctrl.tab[j] = (int16_t)resident_slot(j, nres, nch);
+      ctrl.ord[j] = (int16_t)o;
+      if (ctrl.tab[j] < 0) ++o;
+    }
     mbar_init(smem_u32(&ctrl.xbar[0]), cl * kNW);
     mbar_init(smem_u32(&ctrl.xbar[1]), cl * kNW);
     mbar_init(smem_u32(&ctrl.sbar), cl * kNW);
@@ -523,7 +556,9 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
     ctrl.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (TM && warp == kProducerWarp) tm_alloc(smem_u32(&ctrl.tmem_base));   // the whole warp
   __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   cluster_sync_all();  // peers' barriers exist before any remote arrive
 
   // pieces of this CTA's slice that fall into chunk j (<= 0 for chunks past the slice end)
@@ -596,12 +631,12 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
         bool wg, wg_next;
         const int64_t r = cur.locate(p, cluster_id + i * plan.num_clusters, wg);
         // first fetch of a chunk that sweep 2 fetches again: keep it in L2; last fetch: let it go
-        emit(r, i == 0 ? 0 : lead, nch, wg ? pol_keep : pol_once);
+        emit(r, i == 0 ? 0 : lead, nch, (wg && !TM) ? pol_keep : pol_once);
         if (i + 1 < my_rows) {
           const int64_t rn = cur.locate(p, cluster_id + (i + 1) * plan.num_clusters, wg_next);
           emit(rn, 0, lead, wg_next ? pol_keep : pol_once);
         }
-        if (wg) emit(r, 0, nch, pol_once);
+        if (wg && !TM) emit(r, 0, nch, pol_once);   // TM: sweep 2 reads tensor memory instead
       }
       // Drain: every copy this CTA issued must have landed before its shared memory goes away.
       int64_t pending = fills < nring ? fills : nring;
@@ -698,6 +733,10 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
     const int grp = warp / kGW;                  // this warp's group: chunks j % kG == grp
     const int gt = tid - grp * kGT;              // thread index inside the group
     const uint32_t toff = (uint32_t)gt * 16u;    // first of this thread's kP pieces in a chunk
+    // this thread's tensor-memory window: its lane, 128 of the 512 columns
+    const uint32_t tm_lane = TM ? ctrl.tmem_base + ((uint32_t)((warp & 3) * 32) << 16) +
+                                      (uint32_t)((warp >> 2) * kTmColsPerThread)
+                                : 0u;
     const int64_t iters = my_rows > 0 ? my_rows + 1 : 0;   // + one exchange for the last norm
     Acc2 a;        // sweep-1 sums; carries the leading chunks of the next row across sweep 2
     a.reset();
@@ -739,6 +778,7 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
         f2_t nrefs = splat2(-ref_s), nreft = splat2(-ref_t), ndref = splat2(-dref);
         for (int v = v0;; ++v) {
           if (v == nch) {
+            if (TM) tm_wait_st();
             // record = { S, A, St, B0, B1, B2, q_prev, 0 }: this warp's sums over its lanes.
             const float v0s = lane_sum(hsum2(a.S)), v1 = lane_sum(hsum2(a.A)), v2 = lane_sum(hsum2(a.St));
             float v3 = 0.f, v4 = 0.f, v5 = 0.f;
@@ -802,6 +842,13 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
             __syncwarp();
             if (lane == 0)
               mbar_arrive(smem_u32(k < 0 ? &ctrl.ring_empty[rc_slot] : &ctrl.res_empty[k]));
+          }
+          if (TM && k < 0 && wgv) {   // park the pieces for sweep 2 (every lane takes part)
+            const int o = ctrl.ord[j];
+#pragma unroll
+            for (int h = 0; h < kP; ++h)
+              if (ADWIN_CHK((o * kP + h) * 8 + 8 <= kTmColsPerThread, p.status))
+                tm_store8(tm_lane + (uint32_t)((o * kP + h) * 8), zr[h], ur[h]);
           }
 #pragma unroll
           for (int h = 0; h < kP; ++h) {
@@ -943,28 +990,38 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
         for (int j = 0; j < nch; ++j) {
           const int k = ctrl.tab[j];
           if (j % kG == grp) {
-            const char* sl;
+            const char* sl = nullptr;
+            const bool from_tm = TM && k < 0;
             if (k >= 0) {
               sl = res_base + (size_t)k * plan.slot_bytes + toff;   // still there since sweep 1
-            } else {
+            } else if (!TM) {
               if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort, plan.wait_limit_ns)) timed_out = true;
               sl = ring_base + (size_t)rc_slot * plan.slot_bytes + toff;
             }
             if (timed_out) break;
             const int np = pieces_in_chunk(j);
             uint4 zr[kP], ur[kP];
+            if (from_tm) {   // back from tensor memory (every lane takes part)
+              const int o = ctrl.ord[j];
 #pragma unroll
-            for (int h = 0; h < kP; ++h) {
-              if (gt + h * kGT < np &&
-                  ADWIN_CHK(k < nres && rc_slot < nring + (nring == 0) &&
-                                toff + (uint32_t)(h * kGT * 16) + 16u <= u_off, p.status)) {
-                zr[h] = *reinterpret_cast<const uint4*>(sl + h * kGT * 16);
-                ur[h] = *reinterpret_cast<const uint4*>(sl + u_off + h * kGT * 16);
+              for (int h = 0; h < kP; ++h)
+                if (ADWIN_CHK((o * kP + h) * 8 + 8 <= kTmColsPerThread, p.status))
+                  tm_load8(tm_lane + (uint32_t)((o * kP + h) * 8), zr[h], ur[h]);
+              tm_wait_ld();
+            } else {
+#pragma unroll
+              for (int h = 0; h < kP; ++h) {
+                if (gt + h * kGT < np &&
+                    ADWIN_CHK(k < nres && rc_slot < nring + (nring == 0) &&
+                                  toff + (uint32_t)(h * kGT * 16) + 16u <= u_off, p.status)) {
+                  zr[h] = *reinterpret_cast<const uint4*>(sl + h * kGT * 16);
+                  ur[h] = *reinterpret_cast<const uint4*>(sl + u_off + h * kGT * 16);
+                }
               }
+              __syncwarp();
+              if (lane == 0)
+                mbar_arrive(smem_u32(k < 0 ? &ctrl.ring_empty[rc_slot] : &ctrl.res_empty[k]));
             }
-            __syncwarp();
-            if (lane == 0)
-              mbar_arrive(smem_u32(k < 0 ? &ctrl.ring_empty[rc_slot] : &ctrl.res_empty[k]));
 #pragma unroll
             for (int h = 0; h < kP; ++h) {
               if (gt + h * kGT < np) {
@@ -1004,14 +1061,14 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
                   store_pairs<TOut, NP>(gthread + (size_t)j * gstep + (size_t)h * kGT * N * sizeof(TOut), G);
               }
             }
-          } else if (k < 0) {
+          } else if (k < 0 && !TM) {
             if (!bounded_wait<false>(smem_u32(&ctrl.ring_full[rc_slot]), rc_phase, abort, plan.wait_limit_ns)) {
               timed_out = true;
               break;
             }
             if (lane == 0) mbar_arrive(smem_u32(&ctrl.ring_empty[rc_slot]));
           }
-          if (k < 0 && ++rc_slot == nring) {
+          if (!TM && k < 0 && ++rc_slot == nring) {
             rc_slot = 0;
             rc_phase ^= 1u;
           }
@@ -1034,7 +1091,15 @@ __global__ void __launch_bounds__(kThreads, 1) kl_staged_kernel(KlParams p, Stag
   }
   // No CTA leaves while a peer may still write into its shared memory or arrive on its barriers.
   __syncwarp();
+  if (TM) asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   cluster_sync_all();
+  if (TM) {
+    __syncthreads();   // every consumer of this CTA is done with tensor memory
+    if (warp == kProducerWarp) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      tm_dealloc(ctrl.tmem_base);
+    }
+  }
 }
 
 // ---------------------------------------------------------------------------- host side
@@ -1060,6 +1125,7 @@ bool plan_for_cluster(int64_t pieces_total, int cl, bool has_grad, StagedPlan& p
   const int64_t nslot = slots_bytes / slot_bytes;
   if (nslot < 2) return false;
   int64_t nres = 0, nring = 0;
+  int tm = 0;
   if (!has_grad) {
     nring = nslot < kMaxRing ? nslot : kMaxRing;   // nothing is read twice
   } else {
@@ -1072,6 +1138,17 @@ bool plan_for_cluster(int64_t pieces_total, int cl, bool has_grad, StagedPlan& p
     nring = nslot - nres;
     if (nring > kMaxRing) nring = kMaxRing;
     if (nres == nch) nring = 0;                    // everything resident: no stream
+    // Tensor-memory mode: the streamed chunks are parked in tensor memory between the sweeps
+    // (kTmColsPerThread / (kP * 8) chunks fit); only the chunks beyond that stay resident in shared
+    // memory and the whole rest of it is a ring that streams from HBM during both sweeps.
+    const int64_t stash = kTmColsPerThread / (kP * 8);
+    const int64_t nres_tm = nch > stash ? nch - stash : 0;
+    if (nres_tm <= nslot - 2 && nres_tm <= kMaxRes && nres_tm < nch) {
+      tm = 1;
+      nres = nres_tm;
+      nring = nslot - nres;
+      if (nring > kMaxRing) nring = kMaxRing;
+    }
   }
   plan.cl = cl;
   plan.nch = (int)nch;
@@ -1082,12 +1159,13 @@ bool plan_for_cluster(int64_t pieces_total, int cl, bool has_grad, StagedPlan& p
     // current row is in flight (at most kLeadMax chunks, and never the whole slice).
     int lead = 0;
     while (lead < kLeadMax && lead + 1 < nch && ((lead + 1) * nres) / nch == (lead * nres) / nch) ++lead;
-    if (nring < 2) lead = 0;
+    if (nring < 2 || tm) lead = 0;   // (tensor-memory mode: the next row's chunks would overwrite this row's)
     plan.lead = lead;
   }
   plan.chunk_pieces = (int)chunk_pieces;
   plan.per_rank_pieces = (int)per_rank;
   plan.slot_bytes = (uint32_t)slot_bytes;
+  plan.tm = tm;
   return true;
 }
 
@@ -1097,7 +1175,7 @@ int plan_smem_bytes(const StagedPlan& plan) {
 
 template <typename TIn, typename TOut>
 cudaError_t max_clusters_for(const StagedPlan& plan, int sm_count, int& max_clusters) {
-  auto kernel = kl_staged_kernel<TIn, TOut>;
+  auto kernel = plan.tm ? kl_staged_kernel<TIn, TOut, true> : kl_staged_kernel<TIn, TOut, false>;
   const int smem = plan_smem_bytes(plan);
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
@@ -1187,7 +1265,7 @@ cudaError_t launch_staged_t(const KlParams& p, int dtype, int grad_dtype, int sm
   }
   if (!ok) return cudaErrorNotSupported;
 
-  auto kernel = kl_staged_kernel<TIn, TOut>;
+  auto kernel = plan.tm ? kl_staged_kernel<TIn, TOut, true> : kl_staged_kernel<TIn, TOut, false>;
   const int smem = plan_smem_bytes(plan);
   e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
