@@ -74,7 +74,7 @@ def measured_peak():
 # ends, a residue bounded by the L2 size that does not grow with the rows, so at full size the
 # writes are taken as the gradient bytes themselves.
 TRAFFIC_READ_BYTES_PER_ROW = 611598
-TRAFFIC_KERNEL_SHA = "18f9a1f9922e75ed"
+TRAFFIC_KERNEL_SHA = "db42947a1cefc367"
 
 
 def recorded_traffic(rows, V):
