@@ -177,6 +177,18 @@ def test_odd_vocab_sizes(V):
     run_and_check(batch, grad_dtype=None)
 
 
+@pytest.mark.parametrize("V", [409600, 1048576])
+def test_vocabulary_beyond_what_tensor_memory_holds(V):
+    """The staged kernel parks the streamed chunks of a row slice in tensor memory between its
+    sweeps when they fit (up to 5 chunks + the resident slots per CTA, with clusters of up to 4);
+    larger rows go back to fetching those chunks a second time through the shared-memory ring.
+    Both sizes here are beyond the limit (the paper-scale vocabulary is inside it)."""
+    batch = synth.make_batch(3, device=DEV, B=1, T=5, V=V)
+    batch.window = torch.tensor([4], dtype=torch.int32, device=DEV)
+    for mode in (api.GRAD_FULL_KL, api.GRAD_SAMPLED):
+        run_and_check(batch, grad_dtype=torch.bfloat16, grad_mode=mode, flags=api.FORCE_STAGED)
+
+
 @pytest.mark.parametrize("path", PATHS)
 def test_padded_row_stride(path):
     B, T, V, ld = 2, 5, 4096, 4096 + 64
