@@ -10,13 +10,17 @@
 
 namespace adwin {
 
-// 128-thread CTAs, one row each, eight pairs of 16-byte loads in flight per thread: small CTAs put
+// 128-thread CTAs, one row each, five pairs of 16-byte loads in flight per thread: small CTAs put
 // many independent rows on an SM, so one row's reduction overlaps the others' streaming (measured on
-// the read-only pass at V = 151 936: 256 threads x 1 load 74 %, 256 x 8 81 %, 512 x 8 79 %,
-// 128 x 16 78 %, 128 x 8 90 % of the measured copy bandwidth).
+// the read-only pass at V = 151 936 with scalar arithmetic: 256 threads x 1 load 74 %, 256 x 8 81 %,
+// 512 x 8 79 %, 128 x 16 78 %, 128 x 8 90 % of the measured copy bandwidth).  With sweep 1 on packed
+// pairs the kernel wants more registers per thread; 5 loads at 5 CTAs per SM (<= 96 registers, no
+// spills) measured best among 4..8 loads x 4..8 CTAs, 3 % faster than the scalar 128 x 8 form both
+// on a cold GPU and in a back-to-back series (where every form runs ~12 % slower).
 constexpr int kGenericThreads = 128;
 constexpr int kGenericWarps = kGenericThreads / 32;
-constexpr int kGenericUnroll = 8;
+constexpr int kGenericUnroll = 5;
+constexpr int kGenericMinBlocks = 5;   // CTAs per SM the register allocation leaves room for
 
 struct BlockScratch {
   float wm[2][kGenericWarps];
@@ -25,6 +29,111 @@ struct BlockScratch {
   RowScalars rs;
   RowTotals tot;
 };
+
+// Sweep 1 on packed fp32 pairs: sm_100 issues add / mul / fma on two fp32 lanes of a 64-bit
+// register pair in one slot, which halves the issue slots of the element-wise part (the sweep is
+// bound by issue slots and the ex2 unit as much as by memory).  Even and odd entries of a piece
+// accumulate separately; fold() adds the two lanes.
+typedef unsigned long long pair_t;
+__device__ __forceinline__ pair_t pair(float lo, float hi) {
+  pair_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpair(pair_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ pair_t pfma(pair_t a, pair_t b, pair_t c) {
+  pair_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ pair_t padd(pair_t a, pair_t b) {
+  pair_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ pair_t pmul(pair_t a, pair_t b) {
+  pair_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ pair_t pex2(pair_t x) {
+  float a, b;
+  unpair(x, a, b);
+  return pair(ex2f(a), ex2f(b));
+}
+__device__ __forceinline__ float psum(pair_t v) {
+  float a, b;
+  unpair(v, a, b);
+  return a + b;
+}
+
+struct PairAcc {
+  float m2s, m2t;                  // running references, as in RowAcc
+  pair_t S, A, B0, B1, B2, St;     // the sums of RowAcc, even / odd entries apart
+  __device__ __forceinline__ void reset() {
+    m2s = -INFINITY;
+    m2t = -INFINITY;
+    S = A = B0 = B1 = B2 = St = 0ull;   // the bit pattern of {0.f, 0.f}
+  }
+  __device__ __forceinline__ RowAcc fold() const {
+    RowAcc a;
+    a.m2s = m2s;
+    a.m2t = m2t;
+    a.S = psum(S);
+    a.A = psum(A);
+    a.B0 = psum(B0);
+    a.B1 = psum(B1);
+    a.B2 = psum(B2);
+    a.St = psum(St);
+    return a;
+  }
+};
+
+// acc_piece<N, true> on pairs (N even).
+template <int N>
+__device__ __forceinline__ void acc_piece_pairs(const float (&z)[N], const float (&u)[N], float dref,
+                                                PairAcc& a) {
+  float zm = z[0], um = u[0];
+#pragma unroll
+  for (int i = 1; i < N; ++i) {
+    zm = fmaxf(zm, z[i]);
+    um = fmaxf(um, u[i]);
+  }
+  const float zl = zm * kLog2e, ul = um * kLog2e;
+  if (zl > a.m2s) {
+    const float f = ex2f(a.m2s - zl);
+    const pair_t F = pair(f, f), F2 = pmul(F, F);
+    a.S = pmul(a.S, F);
+    a.A = pmul(a.A, F);
+    a.B0 = pmul(a.B0, F2);
+    a.B1 = pmul(a.B1, F2);
+    a.B2 = pmul(a.B2, F2);
+    a.m2s = zl;
+  }
+  if (ul > a.m2t) {
+    const float f = ex2f(a.m2t - ul);
+    a.St = pmul(a.St, pair(f, f));
+    a.m2t = ul;
+  }
+  const pair_t L2 = pair(kLog2e, kLog2e), NEG1 = pair(-1.f, -1.f);
+  const pair_t nms = pair(-a.m2s, -a.m2s), nmt = pair(-a.m2t, -a.m2t), ndref = pair(-dref, -dref);
+#pragma unroll
+  for (int i = 0; i < N; i += 2) {
+    const pair_t Z = pair(z[i], z[i + 1]), U = pair(u[i], u[i + 1]);
+    const pair_t E = pex2(pfma(Z, L2, nms));
+    const pair_t D = padd(pfma(U, NEG1, Z), ndref);
+    a.S = padd(a.S, E);
+    a.A = pfma(E, D, a.A);
+    const pair_t E2 = pmul(E, E);
+    const pair_t E2D = pmul(E2, D);
+    a.B0 = padd(a.B0, E2);
+    a.B1 = padd(a.B1, E2D);
+    a.B2 = pfma(E2D, D, a.B2);
+    a.St = padd(a.St, pex2(pfma(U, L2, nmt)));
+  }
+}
 
 // Combine the per-thread accumulators of a CTA; every thread returns the same totals.
 __device__ __forceinline__ RowTotals block_combine(const RowAcc& a, BlockScratch& sm) {
@@ -74,7 +183,7 @@ __device__ __forceinline__ RowTotals block_combine(const RowAcc& a, BlockScratch
 }
 
 template <typename TIn, typename TOut, bool VEC>
-__global__ void __launch_bounds__(kGenericThreads) kl_generic_kernel(KlParams p) {
+__global__ void __launch_bounds__(kGenericThreads, kGenericMinBlocks) kl_generic_kernel(KlParams p) {
   __shared__ BlockScratch sm;
   constexpr int N = VEC ? Elem<TIn>::N : 1;
   const int64_t rows = p.B * p.T;
@@ -99,6 +208,8 @@ __global__ void __launch_bounds__(kGenericThreads) kl_generic_kernel(KlParams p)
     a.reset();
     const int64_t pieces = (p.V + N - 1) / N;  // VEC requires V % N == 0
     if (VEC) {
+      PairAcc pa;
+      pa.reset();
       // kGenericUnroll pairs of 16-byte loads in flight per thread; a row that is read only once
       // (no gradient) is streamed past the caches, otherwise sweep 2 should find it in L2
       const uint4* zs = reinterpret_cast<const uint4*>(zrow);
@@ -118,7 +229,7 @@ __global__ void __launch_bounds__(kGenericThreads) kl_generic_kernel(KlParams p)
           float z[N], u[N];
           Elem<TIn>::unpack(zv[h], reinterpret_cast<float(&)[Elem<TIn>::N]>(z));
           Elem<TIn>::unpack(uv[h], reinterpret_cast<float(&)[Elem<TIn>::N]>(u));
-          acc_piece<N, true>(z, u, dref, a);
+          acc_piece_pairs<N>(z, u, dref, pa);
         }
       }
       for (; i < pieces; i += kGenericThreads) {
@@ -128,8 +239,9 @@ __global__ void __launch_bounds__(kGenericThreads) kl_generic_kernel(KlParams p)
         const uint4 uv = write_grad ? __ldg(us + i) : __ldcs(us + i);
         Elem<TIn>::unpack(zv, reinterpret_cast<float(&)[Elem<TIn>::N]>(z));
         Elem<TIn>::unpack(uv, reinterpret_cast<float(&)[Elem<TIn>::N]>(u));
-        acc_piece<N, true>(z, u, dref, a);
+        acc_piece_pairs<N>(z, u, dref, pa);
       }
+      a = pa.fold();
     } else {
       for (int64_t i = tid; i < pieces; i += kGenericThreads) {
         float z[N], u[N];
